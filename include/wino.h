@@ -1,0 +1,182 @@
+/*
+ * wino.h - C ABI of the B200 (sm_100a) Winograd-aware quantized 3x3 convolution
+ * forward pass.
+ *
+ * The layer computes, for every (m+2)x(m+2) input patch d and 3x3 filter g,
+ *     Y = A^T [ (G g G^T) (.) (B^T d B) ] A            (paper: Section 3.1, Eq. 1)
+ * with a uniform quantizer after every stage (paper: Fig. 2 and Section 3.2:
+ * transformed weights, transformed input, Hadamard product, output) using
+ * per-layer symmetric quantization (paper: Section 5.1).  The transform
+ * matrices B^T, G, A^T are data: either the Cook-Toom ones or relaxed, learnt
+ * ("flex") ones (paper: Sections 3.1, 3.2).
+ *
+ * Notation.  t = m + 2; xi = i*t + j indexes the t*t Winograd-domain positions;
+ * TH = ceil(H/m), TW = ceil(W/m), T = N*TH*TW tiles; tile index
+ * tau = (n*TH + th)*TW + tw.  Filters are 3x3, stride 1, zero padding 1.
+ *
+ * Tensor layouts (dense, row-major in the index order written, DEVICE memory):
+ *   x    int8  [N][H][W][C]      activations (codes)
+ *   w    int8  [K][3][3][C]      filters (codes)
+ *   U_q  int8  [t*t][K][C]       transformed, quantized filters
+ *   y    int8 or float [N][H][W][K]
+ *   bias float [K]               in real units (optional)
+ *
+ * Arithmetic contract (what "the same result" means, bit for bit):
+ *   - quantizer  Q(v; mult, z, qmin, qmax) = clamp(rne(v * mult) + z, qmin, qmax)
+ *     with one fp32 multiply, round-half-to-even, and mult a precomputed fp32:
+ *     mult = (float)((double)s_src / (double)s_dst);
+ *   - a transform  Z = (L X) L^T  is evaluated as a left pass then a right pass,
+ *     each entry one fused-multiply-add chain starting from 0.0f and running
+ *     over the contracted index in ascending order, in fp32;
+ *   - input stage   V = B^T d B on d = (float)(x - z_x) (0 outside the image),
+ *                   V_q = Q(V; s_x/s_V);
+ *   - weight stage  U = G g G^T on g = (float)(w - z_w), U_q = Q(U; s_w/s_U);
+ *   - Hadamard stage M[xi][tau][k] = sum_c V_q * U_q in int32 (exact),
+ *                   m_q = Q((float)M; s_U*s_V/s_M) when q_M.enabled;
+ *   - output stage  right factor first: R = m A, then Y = A^T R (same chain
+ *                   rule), m = (float)m_q, or (float)M when q_M is disabled;
+ *                   int8 output: Q(fmaf(Y, s_acc/s_Y, bias/s_Y); 1) with
+ *                   s_acc = s_M (or s_U*s_V when q_M is disabled);
+ *                   float output: fmaf(Y, (float)s_acc, bias).
+ *
+ * Ownership.  The caller owns every device buffer and the stream.  A plan owns
+ * only its copy of the descriptor and matrices plus one small device status
+ * word.  No entry point below allocates device memory except wino_plan.
+ *
+ * Errors.  Every function returns WINO_OK (0) or a negative code; nothing
+ * throws, aborts or traps.  Launches are asynchronous on the given stream.
+ */
+#ifndef WINO_H_
+#define WINO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  WINO_OK = 0,
+  WINO_ERR_INVALID = -1,     /* null pointer, size out of range, bad enum */
+  WINO_ERR_UNSUPPORTED = -2, /* valid request this build does not implement */
+  WINO_ERR_ALIGNMENT = -3,   /* a device pointer is not 16-byte aligned */
+  WINO_ERR_WORKSPACE = -4,   /* workspace missing */
+  WINO_ERR_CUDA = -5,        /* a CUDA runtime / driver call failed */
+  WINO_ERR_TIMEOUT = -6      /* a bounded device-side wait expired */
+};
+
+/* Execution paths a plan can use (see wino_plan_path / wino_plan_force_path). */
+enum {
+  WINO_PATH_AUTO = 0,
+  WINO_PATH_STAGED_TC = 1,   /* transform kernels + tcgen05 int8 GEMMs */
+  WINO_PATH_STAGED_DP4A = 2, /* transform kernels + integer-dot-product GEMMs on the ALUs */
+  WINO_PATH_SMALLC = 3       /* one fused warp-shuffle kernel, C <= 32 and K <= 32 */
+};
+
+/* Stages that wino_debug_dump_stage can copy out (staged paths only). */
+enum { WINO_STAGE_VQ = 0, WINO_STAGE_M_I32 = 1, WINO_STAGE_MQ = 2 };
+
+/* One uniform quantizer (paper: Section 5.1).  real = scale * (code - zero_point);
+ * codes are clamped to [qmin, qmax], which must lie inside [-128, 127].
+ * `enabled` is only read for q_M (0 = feed the int32 sums straight to the output
+ * transform). */
+typedef struct {
+  float scale;
+  int32_t zero_point;
+  int32_t qmin, qmax;
+  int32_t enabled;
+} wino_quant_t;
+
+/* Problem statement of one layer.  BT, G, AT are HOST pointers to row-major
+ * fp32 matrices BT[t][t], G[t][3], AT[m][t]; they are copied by wino_plan.
+ * transforms_exact = 1 is the caller's promise that BT and AT are the Cook-Toom
+ * matrices for the standard points, whose products with integer codes are exact
+ * in fp32 (the library may then reorder sums; results are unchanged).
+ * out_dtype: 0 = int8 codes, 1 = float real values.
+ * Restrictions (WINO_ERR_UNSUPPORTED otherwise): m in {2, 4, 6};
+ * zero_point == 0 for q_V, q_U, q_M; C <= 1040 (so that (float)M is exact). */
+typedef struct {
+  int32_t N, C, H, W, K, m;
+  const float* BT;
+  const float* G;
+  const float* AT;
+  int32_t transforms_exact;
+  wino_quant_t q_x, q_w, q_V, q_U, q_M, q_Y;
+  int32_t out_dtype;
+} wino_desc_t;
+
+typedef struct wino_plan wino_plan_t; /* opaque */
+
+/* Validates the descriptor, copies it, precomputes the fixed multipliers and
+ * picks an execution path (paper: Eq. 1 / Fig. 2 define what is planned).
+ * *out receives a new plan (free with wino_destroy).  Works without a GPU for
+ * size queries; launches then fail with WINO_ERR_CUDA. */
+int wino_plan(const wino_desc_t* desc, wino_plan_t** out);
+
+/* Bytes of U_q: t*t*K*C (paper: Section 3.1 "Memory": 1.78x / 4x the filters). */
+size_t wino_weight_bytes(const wino_plan_t* plan);
+
+/* Bytes of scratch wino_conv_forward needs for the plan's path (V_q and m_q or
+ * M for the staged paths; 0 for the fused small-channel path). */
+size_t wino_workspace_bytes(const wino_plan_t* plan);
+
+/* The path the plan will run (one of WINO_PATH_*), and a way to pin it.
+ * Forcing a path the shape cannot use returns WINO_ERR_UNSUPPORTED. */
+int wino_plan_path(const wino_plan_t* plan);
+int wino_plan_force_path(wino_plan_t* plan, int path);
+
+/* The five fixed multipliers the plan uses, for inspection:
+ * out[0]=s_x/s_V, out[1]=s_w/s_U, out[2]=s_U*s_V/s_M, out[3]=s_acc/s_Y, out[4]=s_acc. */
+int wino_plan_multipliers(const wino_plan_t* plan, float out[5]);
+
+/* Weight transform U_q = Q(G g G^T) (paper: Eq. 1; done once per layer, "amortized
+ * across inferences", Section 3.1).  w_KRSC_dev: int8 [K][3][3][C]; Uq_dev:
+ * int8 [t*t][K][C]; both device pointers, 16-byte aligned.  absmax_dev
+ * (nullable, device, one uint32 holding float bits, caller-zeroed) receives
+ * max |U| before quantization, for calibration. */
+int wino_transform_weights(const wino_plan_t* plan, const int8_t* w_KRSC_dev, int8_t* Uq_dev,
+                           uint32_t* absmax_dev, void* stream);
+
+/* The forward pass (paper: Eq. 1 with the quantizers of Fig. 2): input
+ * transform, Hadamard stage as t*t int8 GEMMs over channels with int32
+ * accumulation, output transform, bias, output quantizer.
+ * x_NHWC_dev int8 [N][H][W][C]; Uq_dev from wino_transform_weights; bias_K_dev
+ * float [K] or NULL; y_NHWK_dev int8 or float [N][H][W][K] per out_dtype;
+ * workspace_dev at least wino_workspace_bytes (may be NULL when that is 0).
+ * All device pointers 16-byte aligned. */
+int wino_conv_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev, const int8_t* Uq_dev,
+                      const float* bias_K_dev, void* y_NHWK_dev, void* workspace_dev,
+                      void* stream);
+
+/* Calibration pass (paper: Table 1 caption, range "warmup"; here a one-shot
+ * max-abs): runs the forward pass on a staged path and records, as float bits
+ * in absmax4_dev[0..3] (device, caller-zeroed uint32[4]), the max-abs of
+ * V (before Q_V), of M (as a float), of Y before the output scaling, and of
+ * the float-mode output fmaf(Y, s_acc, bias).  y_NHWK_dev may be NULL. */
+int wino_calibrate_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev,
+                           const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
+                           void* workspace_dev, uint32_t* absmax4_dev, void* stream);
+
+/* Synchronizes `stream` and returns the plan's device status word: WINO_OK, or
+ * WINO_ERR_TIMEOUT if a bounded wait inside a kernel expired (the kernel then
+ * stopped early and its output is undefined), or WINO_ERR_CUDA. */
+int wino_last_status(const wino_plan_t* plan, void* stream);
+
+/* Copies one intermediate of the most recent wino_conv_forward on this plan
+ * (staged paths only) into dst_dev: V_q int8 [t*t][T][C], M int32 [t*t][T][K]
+ * (recomputed from V_q and U_q with the plan's GEMM kernel), m_q int8
+ * [t*t][T][K].  `bytes` must equal the stage size.  Asynchronous on the stream
+ * of that forward call. */
+int wino_debug_dump_stage(const wino_plan_t* plan, int stage, void* dst_dev, size_t bytes);
+
+/* Number of kernels launched by this plan since it was created. */
+long wino_launch_count(const wino_plan_t* plan);
+
+void wino_destroy(wino_plan_t* plan);
+const char* wino_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WINO_H_ */

@@ -1,0 +1,134 @@
+// Shared device-side definitions for the Winograd-aware quantized convolution
+// kernels (sm_100a).  Notation follows the paper's Eq. 1: B^T, G, A^T are the
+// input, filter and output transform matrices; t = m + 2.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace wino {
+
+constexpr int kMaxT = 8;
+
+// Everything a kernel needs to know about one layer; passed by value as a
+// __grid_constant__ kernel parameter so that matrix entries are constant-bank
+// operands.
+struct Params {
+  int N, C, H, W, K, m, t, TH, TW;
+  int T;                       // tiles: N * TH * TW
+  float BT[kMaxT * kMaxT];     // [t][t]
+  float G[kMaxT * 3];          // [t][3]
+  float AT[6 * kMaxT];         // [m][t]
+  float mult_V, mult_U, mult_M, mult_Y, s_acc;
+  float lo_V, hi_V, lo_U, hi_U, lo_M, hi_M, lo_Y, hi_Y;  // clamp bounds minus zero point
+  int z_x, z_w, z_Y;
+  int qM_enabled;
+  int out_dtype;               // 0 int8, 1 float
+};
+
+// 1.5 * 2^23: adding it to a float of magnitude < 2^22 leaves the
+// round-half-to-even integer in the low mantissa bits.
+constexpr float kMagic = 12582912.0f;
+constexpr int kMagicBits = 0x4B400000;
+
+// Quantizer core: one fp32 multiply, clamp, round half to even.  Returns the
+// float kMagic + code; low byte of its bit pattern is the two's-complement code.
+// Clamping before rounding equals rounding before clamping because the bounds
+// are integers and rounding is monotone.
+__device__ __forceinline__ float quant_magic(float v, float mult, float lo, float hi) {
+  float s = __fmul_rn(v, mult);
+  s = fminf(fmaxf(s, lo), hi);
+  return __fadd_rn(s, kMagic);
+}
+__device__ __forceinline__ int magic_to_int(float r) { return __float_as_int(r) - kMagicBits; }
+__device__ __forceinline__ float magic_to_float(float r) { return __fsub_rn(r, kMagic); }
+
+// int8 byte `sel` (0..3) of a packed word, minus zero point z, as an exact float:
+// flip the sign bit (value + 128 as unsigned), splice into the mantissa of 2^23,
+// subtract 2^23 + 128 + z.
+// `bias` is the float 8388608 + 128 + z (an exact integer).
+__device__ __forceinline__ float byte_to_float(uint32_t word_flipped, int sel, float bias) {
+  uint32_t b = __byte_perm(word_flipped, 0x4B000000u, 0x7440u | (uint32_t)sel);
+  return __fsub_rn(__uint_as_float(b), bias);
+}
+
+__device__ __forceinline__ void atomic_absmax(unsigned* addr, float v) {
+  // non-negative floats order like their bit patterns
+  float m = v;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if ((threadIdx.x & 31) == 0) atomicMax(addr, __float_as_uint(m));
+}
+
+// ---------------------------------------------------------------------------
+// Cook-Toom matrices for the standard points {0, +-1}, {0, +-1, +-2},
+// {0, +-1, +-2, +-1/2} (monic B^T rows, 1/N_j carried by G).  When a plan's
+// matrices equal these bit for bit, kernels are instantiated with the entries
+// as compile-time constants, so zero entries cost nothing.  Skipping a zero
+// coefficient leaves a fused-multiply-add chain's value unchanged.
+// ---------------------------------------------------------------------------
+template <int M> __host__ __device__ constexpr float std_bt(int i, int k);
+template <int M> __host__ __device__ constexpr float std_at(int i, int k);
+
+template <> __host__ __device__ constexpr float std_bt<2>(int i, int k) {
+  constexpr float a[4][4] = {{1, 0, -1, 0}, {0, 1, 1, 0}, {0, -1, 1, 0}, {0, -1, 0, 1}};
+  return a[i][k];
+}
+template <> __host__ __device__ constexpr float std_at<2>(int i, int k) {
+  constexpr float a[2][4] = {{1, 1, 1, 0}, {0, 1, -1, 1}};
+  return a[i][k];
+}
+template <> __host__ __device__ constexpr float std_bt<4>(int i, int k) {
+  constexpr float a[6][6] = {{4, 0, -5, 0, 1, 0},  {0, 4, 4, -1, -1, 0}, {0, -4, 4, 1, -1, 0},
+                             {0, -2, -1, 2, 1, 0}, {0, 2, -1, -2, 1, 0}, {0, 4, 0, -5, 0, 1}};
+  return a[i][k];
+}
+template <> __host__ __device__ constexpr float std_at<4>(int i, int k) {
+  constexpr float a[4][6] = {{1, 1, 1, 1, 1, 0}, {0, 1, -1, 2, -2, 0}, {0, 1, 1, 4, 4, 0},
+                             {0, 1, -1, 8, -8, 1}};
+  return a[i][k];
+}
+template <> __host__ __device__ constexpr float std_bt<6>(int i, int k) {
+  constexpr float a[8][8] = {{1, 0, -5.25f, 0, 5.25f, 0, -1, 0},
+                             {0, -1, -1, 4.25f, 4.25f, -1, -1, 0},
+                             {0, 1, -1, -4.25f, 4.25f, 1, -1, 0},
+                             {0, 0.5f, 0.25f, -2.5f, -1.25f, 2, 1, 0},
+                             {0, -0.5f, 0.25f, 2.5f, -1.25f, -2, 1, 0},
+                             {0, 2, 4, -2.5f, -5, 0.5f, 1, 0},
+                             {0, -2, 4, 2.5f, -5, -0.5f, 1, 0},
+                             {0, -1, 0, 5.25f, 0, -5.25f, 0, 1}};
+  return a[i][k];
+}
+template <> __host__ __device__ constexpr float std_at<6>(int i, int k) {
+  constexpr float a[6][8] = {{1, 1, 1, 1, 1, 1, 1, 0},
+                             {0, 1, -1, 2, -2, 0.5f, -0.5f, 0},
+                             {0, 1, 1, 4, 4, 0.25f, 0.25f, 0},
+                             {0, 1, -1, 8, -8, 0.125f, -0.125f, 0},
+                             {0, 1, 1, 16, 16, 0.0625f, 0.0625f, 0},
+                             {0, 1, -1, 32, -32, 0.03125f, -0.03125f, 1}};
+  return a[i][k];
+}
+
+template <int M, bool STD>
+struct Mat {
+  static constexpr int T = M + 2;
+  __device__ __forceinline__ static float bt(const Params& p, int i, int k) {
+    if constexpr (STD) return std_bt<M>(i, k);
+    else return p.BT[i * T + k];
+  }
+  __device__ __forceinline__ static float at(const Params& p, int i, int k) {
+    if constexpr (STD) return std_at<M>(i, k);
+    else return p.AT[i * T + k];
+  }
+};
+
+// One step of a fused-multiply-add chain; with a compile-time zero coefficient
+// the step disappears (the chain's value is unchanged by it).
+template <bool STD>
+__device__ __forceinline__ float chain(float coef, float x, float acc) {
+  if constexpr (STD) {
+    if (coef == 0.0f) return acc;
+  }
+  return __fmaf_rn(coef, x, acc);
+}
+
+}  // namespace wino

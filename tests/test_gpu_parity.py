@@ -1,0 +1,143 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU
+oracle, element by element on the same seeded inputs.  Integer stages and int8
+outputs must be bit-exact; float outputs within 1e-4 of the output's max
+magnitude (they are in fact expected to be identical)."""
+import numpy as np
+import pytest
+
+import oracle
+import wino_inputs as wi
+from helpers import build_layer, small
+
+pytestmark = pytest.mark.gpu
+
+TC, DP4A, SMALLC = 1, 2, 3
+
+
+def _compare(L, x_q, w_q, bias, path, dumps=True):
+    from gpu_helpers import gpu_run
+    y_ref, d_ref = oracle.forward(L, x_q, w_q, bias=bias, dumps=True)
+    g = gpu_run(L, x_q, w_q, bias, path=path, dumps=dumps)
+    assert g["path"] == path
+    assert (g["U_q"] == d_ref["U_q"]).all(), "U_q"
+    if dumps:
+        assert (g["V_q"] == d_ref["V_q"]).all(), "V_q"
+        assert (g["M"] == d_ref["M"]).all(), "M"
+        if L.q_M.enabled:
+            assert (g["m_q"] == d_ref["m_q"]).all(), "m_q"
+    if L.out_dtype == 0:
+        bad = np.count_nonzero(g["y"] != y_ref)
+        assert bad == 0, f"y differs in {bad} of {y_ref.size}"
+    else:
+        tol = 1e-4 * max(float(np.abs(y_ref).max()), 1e-30)
+        assert float(np.abs(g["y"] - y_ref).max()) <= tol
+    return g
+
+
+SHAPES = [
+    # N, C, H, W, K
+    (1, 16, 8, 8, 16),
+    (2, 32, 7, 9, 48),       # ragged tiles, K not a multiple of 32
+    (3, 64, 13, 5, 64),
+    (1, 160, 6, 6, 80),      # C spans two 128-byte stages with a partial one
+    (5, 48, 10, 11, 272),    # K > 256: two column blocks
+]
+
+
+@pytest.mark.parametrize("m", [2, 4, 6])
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("path", [TC, DP4A])
+def test_staged_paths_every_stage(m, shape, path):
+    N, C, H, W, K = shape
+    wl = wi.Workload("s", 3000 + m, N, C, H, W, K, m)
+    L, x_q, w_q, bias = build_layer(wl)
+    _compare(L, x_q, w_q, bias, path)
+
+
+@pytest.mark.parametrize("m", [2, 4, 6])
+@pytest.mark.parametrize("path", [TC, DP4A, SMALLC])
+def test_flex_matrices(m, path):
+    wl = wi.Workload("f", 3100 + m, 2, 32, 9, 7, 32, m, flex=True)
+    L, x_q, w_q, bias = build_layer(wl)
+    _compare(L, x_q, w_q, bias, path, dumps=path != SMALLC)
+
+
+@pytest.mark.parametrize("m", [2, 4, 6])
+@pytest.mark.parametrize("path", [TC, DP4A, SMALLC])
+@pytest.mark.parametrize("variant", ["no_qm", "float_out", "no_qm_float", "relu", "no_bias", "zero_points"])
+def test_variants(m, path, variant):
+    wl = wi.Workload("v", 3200 + m, 2, 16, 8, 10, 32, m)
+    kw = {}
+    if variant in ("no_qm", "no_qm_float"):
+        kw["q_M"] = False
+    if variant in ("float_out", "no_qm_float"):
+        kw["out_dtype"] = 1
+    if variant == "relu":
+        kw["relu"] = True
+    if variant == "no_bias":
+        kw["with_bias"] = False
+    L, x_q, w_q, bias = build_layer(wl, **kw)
+    if variant == "zero_points":
+        L.q_x.zero_point = 5
+        L.q_w.zero_point = -3
+        L.q_Y.zero_point = 7
+    _compare(L, x_q, w_q, bias, path, dumps=path != SMALLC)
+
+
+@pytest.mark.parametrize("shape", [(1, 4, 3, 3, 4), (2, 8, 1, 1, 12), (1, 32, 5, 20, 32), (7, 20, 6, 6, 28)])
+@pytest.mark.parametrize("m", [2, 4, 6])
+def test_small_channel_path(m, shape):
+    N, C, H, W, K = shape
+    wl = wi.Workload("c", 3300 + m, N, C, H, W, K, m)
+    L, x_q, w_q, bias = build_layer(wl)
+    _compare(L, x_q, w_q, bias, SMALLC, dumps=False)
+    _compare(L, x_q, w_q, bias, DP4A, dumps=True)
+
+
+def test_saturating_scales_clip_identically():
+    wl = wi.Workload("sat", 3400, 2, 32, 8, 8, 32, 4)
+    L, x_q, w_q, bias = build_layer(wl)
+    for q in (L.q_V, L.q_U, L.q_M, L.q_Y):
+        q.scale = q.scale / 7.0           # most values clip
+    g = _compare(L, x_q, w_q, bias, TC)
+    assert np.abs(g["V_q"]).max() == 127 and (np.abs(g["V_q"]) == 127).mean() > 0.05
+
+
+# --- the five workload configurations -------------------------------------------------
+def test_cfg1_all_paths():
+    wl = wi.CONFIGS["cfg1"]
+    L, x_q, w_q, bias = build_layer(wl)
+    for path in (SMALLC, TC, DP4A):
+        _compare(L, x_q, w_q, bias, path, dumps=path != SMALLC)
+
+
+@pytest.mark.parametrize("name", ["cfg2", "cfg3", "cfg4"])
+def test_full_size_configs(name):
+    wl = wi.CONFIGS[name]
+    L, x_q, w_q, bias = build_layer(wl)
+    g = _compare(L, x_q, w_q, bias, TC)
+    assert g["launches"] >= 4
+
+
+def test_cfg3_without_qm():
+    wl = small(wi.CONFIGS["cfg3"], N=32)
+    L, x_q, w_q, bias = build_layer(wl, q_M=False)
+    _compare(L, x_q, w_q, bias, TC)
+
+
+def test_gpu_calibration_matches_oracle_calibration():
+    from paper_2002_10711_b200 import binding
+    from paper_2002_10711_b200.layer import calibrate
+    for name, N in (("cfg2", 2), ("cfg3", 8), ("cfg4", 2)):
+        wl = small(wi.CONFIGS[name], N=N)
+        L, x_q, w_q, bias = build_layer(wl)
+
+        def make_plan(s_V, s_U, s_M, s_Y):
+            import copy
+            L2 = copy.deepcopy(L)
+            L2.q_V.scale, L2.q_U.scale, L2.q_M.scale, L2.q_Y.scale = s_V, s_U, s_M, s_Y
+            return binding.Plan.from_layer(L2)
+
+        got = calibrate(make_plan, x_q, w_q, bias, L.q_x.scale, L.q_w.scale)
+        want = (L.q_V.scale, L.q_U.scale, L.q_M.scale, L.q_Y.scale)
+        assert tuple(np.float32(got)) == tuple(np.float32(want)), (name, got, want)
