@@ -1,0 +1,416 @@
+#!/usr/bin/env python
+"""Benchmark of the Winograd-aware quantized conv forward pass on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one forward pass of the layer (input transform, Hadamard-stage
+GEMMs, output transform, all quantizers) over one batch of the workload, with
+the transformed weights resident, as the paper treats them (Section 3.1: the
+weight transform is amortized across inferences); the weight transform is timed
+separately and reported beside it.  The metric is effective direct-convolution-
+equivalent int8 TOPS: 2*N*H*W*K*C*9 operations per step over the measured time.
+
+Prints ONE JSON line (rank 0).  With torchrun (N > 1) every rank processes its
+own batch (weak scaling, no collective on the data path); time is the max over
+ranks, value the sum of work over that time.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import wino_inputs as wi  # noqa: E402
+
+METRIC = "effective direct-conv-equivalent int8 TOPS (Winograd-aware quantized 3x3 conv forward)"
+UNIT = "TOPS"
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+def direct_ops(wl, N):
+    return 2.0 * N * wl.H * wl.W * wl.K * wl.C * 9
+
+
+def wino_ops(wl, N):
+    t = wl.m + 2
+    T = N * (-(-wl.H // wl.m)) * (-(-wl.W // wl.m))
+    return 2.0 * T * t * t * wl.C * wl.K
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed
+    region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [v.strip() for v in ln.split(",")]
+            if len(f) < 8:
+                continue
+            try:
+                sm.append(float(f[0])); smax.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------
+def run_reference(args, wl):
+    """The CPU oracle, as it stands, on the host cores (rank 0 only)."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    import oracle
+    from helpers import build_layer
+    L, x_q, w_q, bias = build_layer(wl)
+    Uq = oracle.weight_stage(L, w_q)
+    for _ in range(min(args.warmup, 2)):
+        oracle.forward(L, x_q, U_q=Uq, bias=bias)
+    steps = min(args.steps, 20)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.forward(L, x_q, U_q=Uq, bias=bias)
+    dt = (time.perf_counter() - t0) / steps
+    value = direct_ops(wl, wl.N) / dt / 1e12
+    cores = oracle.num_threads()
+    sample = f"full batch N={wl.N} per step, {steps} steps"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": min(args.warmup, 2), "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+        "data": "synthetic", "config": workload_config(wl, "host memory (CPU oracle)"),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(wl, l2_note):
+    return {"workload": f"{wl.name}: ResNet-18 CIFAR layer N={wl.N} C=K={wl.C} H=W={wl.H} "
+                        f"F({wl.m}x{wl.m},3x3) int8, per-stage max-abs scales",
+            "N": wl.N, "C": wl.C, "K": wl.K, "H": wl.H, "W": wl.W, "m": wl.m, "l2": l2_note}
+
+
+def aggregate(ms_local: float, units_local: float, dist=None):
+    """Max time over ranks, summed work.  `dist`: torch.distributed or None."""
+    if dist is None or not dist.is_initialized() or dist.get_world_size() == 1:
+        return ms_local, units_local
+    import torch
+    dev = "cuda" if dist.get_backend() == "nccl" else "cpu"
+    t = torch.tensor([ms_local], dtype=torch.float64, device=dev)
+    u = torch.tensor([units_local], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+def run_ours(args, wl):
+    import torch
+    import torch.distributed as dist
+    from paper_2002_10711_b200 import binding, cook_toom
+    from paper_2002_10711_b200.layer import calibrate
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+
+    # ---- inputs: seeded, synthetic; every rank draws its own batch ----
+    wl_r = wi.Workload(**{**wl.__dict__, "seed": wl.seed + 7919 * rank})
+    x_q, s_x, w_q, s_w, bias = wi.make_tensors(wl_r)
+    BT, G, AT = cook_toom(wl.m)
+    if wl.flex:
+        BT = wi.flex_perturb(BT, wl.seed, wi.S_BT)
+        G = wi.flex_perturb(G, wl.seed, wi.S_G)
+        AT = wi.flex_perturb(AT, wl.seed, wi.S_AT)
+    q = lambda s, **kw: dict(scale=float(s), **kw)
+
+    def make_plan(s_V, s_U, s_M, s_Y):
+        return binding.Plan(wl.N, wl.C, wl.H, wl.W, wl.K, wl.m, BT, G, AT, q(s_x), q(s_w), q(s_V),
+                            q(s_U), q(s_M), q(s_Y), out_dtype=0)
+
+    s_V, s_U, s_M, s_Y = calibrate(make_plan, x_q, w_q, bias, s_x, s_w, device=dev)
+    plan = make_plan(s_V, s_U, s_M, s_Y)
+
+    # ---- device buffers: R rotating sets so that x, y and U_q come from HBM ----
+    xb = x_q.nbytes
+    yb = wl.N * wl.H * wl.W * wl.K
+    R = max(4, int(np.ceil(2 * 126e6 / (xb + yb + plan.weight_bytes))))
+    x0 = torch.from_numpy(x_q).to(dev)
+    w_dev = torch.from_numpy(w_q).to(dev)
+    b_dev = torch.from_numpy(bias).to(dev)
+    xs = [x0.clone() for _ in range(R)]
+    ys = [torch.empty((wl.N, wl.H, wl.W, wl.K), dtype=torch.int8, device=dev) for _ in range(R)]
+    Us = [torch.empty(plan.weight_bytes, dtype=torch.int8, device=dev) for _ in range(R)]
+    ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device=dev)
+    for U in Us:
+        plan.transform_weights(w_dev, U)
+    torch.cuda.synchronize()
+
+    def step(i):
+        j = i % R
+        plan.conv_forward(xs[j], Us[j], b_dev, ys[j], ws)
+
+    # ---- warm-up (also sets kernel attributes before any capture) ----
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    torch.cuda.synchronize()
+    assert plan.last_status() == 0
+
+    chunk = min(args.steps, 2 * R)
+    side = torch.cuda.Stream(device=dev)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for i in range(chunk):
+                step(i)
+    torch.cuda.synchronize()
+    launches_per_step = 3 if plan.path != binding.PATH_SMALLC else 1
+    graph.replay()
+    torch.cuda.synchronize()
+
+    # ---- timed region ----
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    replays, rem = divmod(args.steps, chunk)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # spin the clocks up for a moment so the timed region does not start cold
+    for _ in range(3):
+        graph.replay()
+    barrier()
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(replays):
+        graph.replay()
+    for i in range(rem):
+        step(i)
+    e1.record()
+    torch.cuda.synchronize()
+    barrier()
+    ms_local = e0.elapsed_time(e1)
+    status = plan.last_status()
+    assert status == 0, binding.strerror(status)
+    ms, units = aggregate(ms_local, direct_ops(wl, wl.N) * args.steps, dist if world > 1 else None)
+    value = units / (ms * 1e-3) / 1e12
+    ms_per_step = ms / args.steps
+
+    # ---- per-kernel times for the roofline: events between the three kernels,
+    #      launches queued behind a short device-side delay so that host launch
+    #      latency is not measured ----
+    peaks = load_peaks()
+    roofline = None
+    stages = None
+    if plan.path != binding.PATH_SMALLC:
+        nprof = 60
+        evs = []
+        for i in range(nprof):
+            four = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+            for e in four:
+                e.record()
+            evs.append(four)
+        torch.cuda.synchronize()
+        for i in range(nprof):
+            plan.set_stage_events([e.cuda_event for e in evs[i]])
+            torch.cuda._sleep(400000)
+            step(i)
+        plan.set_stage_events(None)
+        torch.cuda.synchronize()
+        dur = [[evs[i][k].elapsed_time(evs[i][k + 1]) * 1e3 for i in range(nprof)] for k in range(3)]
+        us = [statistics.median(d) for d in dur]
+        t = wl.m + 2
+        T = plan.T
+        vq = t * t * T * wl.C
+        mq = t * t * T * wl.K
+        alg = {"input_transform": xb + vq, "hadamard_gemm": vq + plan.weight_bytes + mq,
+               "output_transform": mq + yb}
+        names = ["input_transform", "hadamard_gemm", "output_transform"]
+        stages = {n: {"us": u, "algorithmic_bytes": alg[n], "GBps": alg[n] / (u * 1e-6) / 1e9}
+                  for n, u in zip(names, us)}
+        stages["hadamard_gemm"]["wino_TOPS"] = wino_ops(wl, wl.N) / (us[1] * 1e-6) / 1e12
+        dom = max(range(3), key=lambda k: us[k])
+        if dom == 1:
+            peak = 2.0 * peaks["bf16_tflops"]
+            ach = wino_ops(wl, wl.N) / (us[1] * 1e-6) / 1e12
+            roofline = {"kernel": "k_gemm_tc", "bound": "tensor", "achieved": ach, "peak": peak,
+                        "unit": "TOP/s", "frac": ach / peak, "traffic": None,
+                        "peak_note": f"int8 = 2 x {peaks['source']} bf16 burst peak"}
+        else:
+            n = names[dom]
+            ach = alg[n] / (us[dom] * 1e-6) / 1e9
+            roofline = {"kernel": "k_" + n, "bound": "hbm", "achieved": ach,
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+                        "traffic": None, "peak_note": f"of {peaks['source']}"}
+    # whole-layer roofline of the path's definition: slower of MMA work at the int8
+    # tensor peak and algorithmic bytes (x + y + U_q) at the HBM peak
+    t_mma = wino_ops(wl, wl.N) / (2.0 * peaks["bf16_tflops"] * 1e12)
+    t_hbm = (xb + yb + plan.weight_bytes) / (peaks["hbm_gbs"] * 1e9)
+    layer_roof = {"t_mma_us": t_mma * 1e6, "t_hbm_us": t_hbm * 1e6,
+                  "roofline_us": max(t_mma, t_hbm) * 1e6,
+                  "frac": max(t_mma, t_hbm) / (ms_local / args.steps * 1e-3),
+                  "peaks": peaks["source"]}
+
+    # ---- weight transform, timed alone ----
+    f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    nw = 50
+    f0.record()
+    for i in range(nw):
+        plan.transform_weights(w_dev, Us[i % R])
+    f1.record()
+    torch.cuda.synchronize()
+    wt_us = f0.elapsed_time(f1) * 1e3 / nw
+    wt_bytes = w_q.nbytes + plan.weight_bytes
+
+    # ---- end to end: pinned host input -> device -> forward -> pinned host output ----
+    xh = [torch.from_numpy(x_q).pin_memory() for _ in range(2)]
+    yh = [torch.empty((wl.N, wl.H, wl.W, wl.K), dtype=torch.int8).pin_memory() for _ in range(2)]
+    ke = min(args.steps, 200)
+
+    def e2e_step(i):
+        j = i % R
+        xs[j].copy_(xh[i % 2], non_blocking=True)
+        plan.conv_forward(xs[j], Us[j], b_dev, ys[j], ws)
+        yh[i % 2].copy_(ys[j], non_blocking=True)
+
+    for i in range(3):
+        e2e_step(i)
+    barrier()
+    torch.cuda.synchronize()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record()
+    for i in range(ke):
+        e2e_step(i)
+    g1.record()
+    torch.cuda.synchronize()
+    barrier()
+    e2e_ms, e2e_units = aggregate(g0.elapsed_time(g1), direct_ops(wl, wl.N) * ke,
+                                  dist if world > 1 else None)
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- the oracle beside it (rank 0, single GPU runs only) ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sys.path.insert(0, os.path.join(ROOT, "tests"))
+        import oracle
+        L = oracle.Layer(wl.N, wl.C, wl.H, wl.W, wl.K, wl.m, BT, G, AT)
+        for qq, s in zip((L.q_x, L.q_w, L.q_V, L.q_U, L.q_M, L.q_Y), (s_x, s_w, s_V, s_U, s_M, s_Y)):
+            qq.scale = float(s)
+        Uq_ref = oracle.weight_stage(L, w_q)
+        y_ref = oracle.forward(L, x_q, U_q=Uq_ref, bias=bias)
+        parity = bool((ys[0].cpu().numpy() == y_ref).all()) if rank == 0 else None
+        nrun = 5
+        t0 = time.perf_counter()
+        for _ in range(nrun):
+            oracle.forward(L, x_q, U_q=Uq_ref, bias=bias)
+        dt = (time.perf_counter() - t0) / nrun
+        cpu = {"value": direct_ops(wl, wl.N) / dt / 1e12, "unit": UNIT,
+               "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"full batch N={wl.N}, mean of {nrun} runs ({dt * 1e3:.0f} ms each)",
+               "parity_with_gpu_output": parity}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+            "config": workload_config(
+                wl, f"inputs rotate over {R} buffer sets ({R * (xb + yb + plan.weight_bytes) / 1e6:.0f} MB > L2)"),
+            "wino_domain_TOPS": wino_ops(wl, wl.N) * world / (ms_per_step * 1e-3) / 1e12,
+            "path": {1: "staged_tc", 2: "staged_dp4a", 3: "smallc"}[plan.path],
+            "gpu_launches": launches_per_step * args.steps,
+            "roofline": roofline, "layer_roofline": layer_roof, "stages": stages,
+            "weight_transform": {"us": wt_us, "GBps": wt_bytes / (wt_us * 1e-6) / 1e9,
+                                 "algorithmic_bytes": wt_bytes},
+            "e2e": {"value": e2e_units / (e2e_ms * 1e-3) / 1e12, "unit": UNIT,
+                    "h2d_bytes_per_step": xb, "d2h_bytes_per_step": yb, "steps": ke},
+            "cpu_baseline": cpu, "clocks": clocks,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg3", choices=sorted(wi.CONFIGS))
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    wl = wi.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, wl)
+    else:
+        run_ours(args, wl)
+
+
+if __name__ == "__main__":
+    main()

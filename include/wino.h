@@ -117,8 +117,9 @@ int wino_plan(const wino_desc_t* desc, wino_plan_t** out);
 /* Bytes of U_q: t*t*K*C (paper: Section 3.1 "Memory": 1.78x / 4x the filters). */
 size_t wino_weight_bytes(const wino_plan_t* plan);
 
-/* Bytes of scratch wino_conv_forward needs for the plan's path (V_q and m_q or
- * M for the staged paths; 0 for the fused small-channel path). */
+/* Bytes of scratch for the staged paths and for wino_calibrate_forward: V_q plus
+ * m_q (or M in int32 when q_M is disabled).  On the fused small-channel path
+ * wino_conv_forward itself needs none and accepts a NULL workspace. */
 size_t wino_workspace_bytes(const wino_plan_t* plan);
 
 /* The path the plan will run (one of WINO_PATH_*), and a way to pin it.
@@ -172,6 +173,13 @@ int wino_debug_dump_stage(const wino_plan_t* plan, int stage, void* dst_dev, siz
 
 /* Number of kernels launched by this plan since it was created. */
 long wino_launch_count(const wino_plan_t* plan);
+
+/* Measurement hook for the staged paths (the stages are those of the paper's
+ * Fig. 2): when set, every wino_conv_forward records the four caller-owned
+ * cudaEvent_t handles on its stream: before the input transform, after it,
+ * after the Hadamard-stage GEMMs, after the output transform.  NULL switches
+ * the hook off.  The fused small-channel path records nothing. */
+int wino_plan_set_stage_events(wino_plan_t* plan, void* const events[4]);
 
 void wino_destroy(wino_plan_t* plan);
 const char* wino_strerror(int code);

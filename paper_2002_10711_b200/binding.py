@@ -23,7 +23,7 @@ EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
     "wino_conv_forward", "wino_calibrate_forward", "wino_last_status", "wino_debug_dump_stage",
-    "wino_launch_count", "wino_destroy", "wino_strerror",
+    "wino_launch_count", "wino_plan_set_stage_events", "wino_destroy", "wino_strerror",
 ]
 
 
@@ -69,6 +69,7 @@ def _load() -> ct.CDLL:
     lib.wino_debug_dump_stage.argtypes = [vp, i32, vp, sz]
     lib.wino_launch_count.argtypes = [vp]
     lib.wino_launch_count.restype = ct.c_long
+    lib.wino_plan_set_stage_events.argtypes = [vp, vp]
     lib.wino_destroy.argtypes = [vp]
     lib.wino_destroy.restype = None
     lib.wino_strerror.argtypes = [i32]
@@ -186,6 +187,16 @@ class Plan:
         _check(_lib.wino_calibrate_forward(self._h, _dptr(x_dev), _dptr(Uq_dev), _dptr(bias_dev),
                                            _dptr(y_dev), _dptr(workspace_dev), _dptr(absmax4_dev),
                                            _stream_handle(stream)), "wino_calibrate_forward")
+
+    def set_stage_events(self, events) -> None:
+        """events: four cudaEvent_t handles (ints), or None to switch the hook off."""
+        if events is None:
+            _check(_lib.wino_plan_set_stage_events(self._h, None), "wino_plan_set_stage_events")
+            return
+        arr = (ct.c_void_p * 4)(*[ct.c_void_p(int(e)) for e in events])
+        self._stage_events = arr
+        _check(_lib.wino_plan_set_stage_events(self._h, ct.cast(arr, ct.c_void_p)),
+               "wino_plan_set_stage_events")
 
     def last_status(self, stream=None) -> int:
         return _lib.wino_last_status(self._h, _stream_handle(stream))

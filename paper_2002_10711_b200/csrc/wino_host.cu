@@ -39,6 +39,8 @@ struct wino_plan {
   mutable void* last_ws;
   mutable cudaStream_t last_stream;
   mutable long launches;
+  cudaEvent_t stage_ev[4];  // caller-owned; recorded around the three staged kernels when set
+  bool stage_ev_on;
 };
 
 namespace {
@@ -223,14 +225,19 @@ int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const
     tmp_holder.path = WINO_PATH_STAGED_DP4A;
     run = &tmp_holder;
   }
+  const bool ev = pl->stage_ev_on;
+  if (ev) cudaEventRecord(pl->stage_ev[0], st);
   int rc = DISPATCH_M(pl, launch_input)(pl, x, Vq, calib ? absmax4 + 0 : nullptr, st);
   if (rc != WINO_OK) return rc;
+  if (ev) cudaEventRecord(pl->stage_ev[1], st);
   rc = launch_gemm(run, Vq, Uq, mbuf, pl->p.qM_enabled ? kOutMq : kOutI32,
                    calib ? absmax4 + 1 : nullptr, st);
   if (run != pl) pl->launches++;
   if (rc != WINO_OK) return rc;
+  if (ev) cudaEventRecord(pl->stage_ev[2], st);
   rc = DISPATCH_M(pl, launch_output)(pl, mbuf, bias, y, calib ? absmax4 + 2 : nullptr, st);
   if (rc != WINO_OK) return rc;
+  if (ev) cudaEventRecord(pl->stage_ev[3], st);
   pl->last_uq = Uq;
   pl->last_ws = ws;
   pl->last_stream = st;
@@ -409,6 +416,17 @@ int wino_debug_dump_stage(const wino_plan_t* pl, int stage, void* dst, size_t by
 }
 
 long wino_launch_count(const wino_plan_t* pl) { return pl ? pl->launches : 0; }
+
+int wino_plan_set_stage_events(wino_plan_t* pl, void* const events[4]) {
+  if (pl == nullptr) return WINO_ERR_INVALID;
+  if (events == nullptr) { pl->stage_ev_on = false; return WINO_OK; }
+  for (int i = 0; i < 4; ++i) {
+    if (events[i] == nullptr) return WINO_ERR_INVALID;
+    pl->stage_ev[i] = (cudaEvent_t)events[i];
+  }
+  pl->stage_ev_on = true;
+  return WINO_OK;
+}
 
 void wino_destroy(wino_plan_t* pl) {
   if (pl == nullptr) return;
