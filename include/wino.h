@@ -69,9 +69,10 @@ enum {
 /* Execution paths a plan can use (see wino_plan_path / wino_plan_force_path). */
 enum {
   WINO_PATH_AUTO = 0,
-  WINO_PATH_STAGED_TC = 1,   /* transform kernels + tcgen05 int8 GEMMs */
+  WINO_PATH_STAGED_TC = 1,   /* transform kernels (TMA-staged where the shape allows) + tcgen05 int8 GEMMs */
   WINO_PATH_STAGED_DP4A = 2, /* transform kernels + integer-dot-product GEMMs on the ALUs */
-  WINO_PATH_SMALLC = 3       /* one fused warp-shuffle kernel, C <= 32 and K <= 32 */
+  WINO_PATH_SMALLC = 3,      /* one fused warp-shuffle kernel, C <= 32 and K <= 32 */
+  WINO_PATH_STAGED_TC_PTR = 4 /* as 1, but always the pointer-based transform kernels */
 };
 
 /* Stages that wino_debug_dump_stage can copy out (staged paths only). */

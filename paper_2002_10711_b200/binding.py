@@ -16,7 +16,7 @@ LIB_PATH = os.path.join(_HERE, "libwino_b200.so")
 
 WINO_OK = 0
 ERR_INVALID, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
-PATH_AUTO, PATH_STAGED_TC, PATH_STAGED_DP4A, PATH_SMALLC = 0, 1, 2, 3
+PATH_AUTO, PATH_STAGED_TC, PATH_STAGED_DP4A, PATH_SMALLC, PATH_STAGED_TC_PTR = 0, 1, 2, 3, 4
 STAGE_VQ, STAGE_M_I32, STAGE_MQ = 0, 1, 2
 
 EXPORTS = [
@@ -143,7 +143,7 @@ class Plan:
 
     def __del__(self):
         h = getattr(self, "_h", None)
-        if h is not None and h.value:
+        if h is not None and h.value and _lib is not None:
             _lib.wino_destroy(h)
             self._h = ct.c_void_p()
 

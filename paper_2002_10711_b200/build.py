@@ -1,35 +1,54 @@
-"""Builds the CUDA library (sm_100a only) in-tree with nvcc."""
+"""Builds the CUDA library (sm_100a only) in-tree with nvcc: one object per
+translation unit, compiled in parallel, linked into one shared library."""
 from __future__ import annotations
 
 import os
 import subprocess
+from concurrent.futures import ThreadPoolExecutor
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
+OBJ = os.path.join(HERE, "_build")
 LIB = os.path.join(HERE, "libwino_b200.so")
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
-    "-fmad=false", "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC", "-shared",
-    "-cudart", "static",
+    "-fmad=false", "--expt-relaxed-constexpr", "-Xcompiler", "-fPIC",
 ]
 
 
-def sources():
-    return sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".cu", ".cuh")))
+def _units():
+    return sorted(f for f in os.listdir(CSRC) if f.endswith(".cu"))
+
+
+def _headers():
+    hs = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith((".h", ".cuh"))]
+    return hs + [os.path.join(ROOT, "include", "wino.h")]
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    newest = max(os.path.getmtime(f) for f in sources() + [os.path.join(ROOT, "include", "wino.h")])
-    if force or not os.path.exists(LIB) or os.path.getmtime(LIB) < newest:
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    os.makedirs(OBJ, exist_ok=True)
+    hdr_time = max(os.path.getmtime(h) for h in _headers())
+    jobs = []
+    for u in _units():
+        src = os.path.join(CSRC, u)
+        obj = os.path.join(OBJ, u[:-3] + ".o")
+        if force or not os.path.exists(obj) or os.path.getmtime(obj) < max(os.path.getmtime(src), hdr_time):
+            cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC, "-c", src, "-o", obj]
+            if verbose:
+                cmd[1:1] = ["-Xptxas", "-v"]
+            jobs.append(cmd)
+    if jobs:
+        with ThreadPoolExecutor(max_workers=min(len(jobs), os.cpu_count() or 4)) as ex:
+            for rc in ex.map(lambda c: subprocess.run(c).returncode, jobs):
+                if rc != 0:
+                    raise RuntimeError("nvcc failed")
+    objs = [os.path.join(OBJ, u[:-3] + ".o") for u in _units()]
+    if jobs or not os.path.exists(LIB) or os.path.getmtime(LIB) < max(os.path.getmtime(o) for o in objs):
         tmp = LIB + f".tmp{os.getpid()}"
-        cmd = [nvcc, *NVCC_FLAGS, "-I", os.path.join(ROOT, "include"), "-I", CSRC,
-               os.path.join(CSRC, "wino_host.cu"), "-o", tmp]
-        if verbose:
-            cmd.insert(1, "-Xptxas")
-            cmd.insert(2, "-v")
-        subprocess.check_call(cmd)
+        subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared",
+                               "-cudart", "static", *objs, "-o", tmp])
         os.replace(tmp, LIB)
     return LIB
 

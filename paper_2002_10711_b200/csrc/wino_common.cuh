@@ -50,6 +50,28 @@ __device__ __forceinline__ float byte_to_float(uint32_t word_flipped, int sel, f
   uint32_t b = __byte_perm(word_flipped, 0x4B000000u, 0x7440u | (uint32_t)sel);
   return __fsub_rn(__uint_as_float(b), bias);
 }
+// Same with a precomputed permute selector (0x7440 | byte index).
+__device__ __forceinline__ float byte_to_float_sel(uint32_t word_flipped, uint32_t selector,
+                                                   float bias) {
+  return __fsub_rn(__uint_as_float(__byte_perm(word_flipped, 0x4B000000u, selector)), bias);
+}
+// Permute selector that inserts byte 0 of the second operand at byte `ch` of the first.
+__device__ __forceinline__ uint32_t insert_selector(int ch) {
+  return (0x3210u & ~(0xFu << (4 * ch))) | (4u << (4 * ch));
+}
+
+// Programmatic dependent launch: wait for the preceding kernel on the stream to
+// finish (no-op when the kernel was launched normally); allow the following
+// kernel to be scheduled early.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
+// Exact int32 -> float for |v| < 2^22 without a conversion instruction.
+__device__ __forceinline__ float small_int_to_float(int v) {
+  return __fsub_rn(__int_as_float(v + kMagicBits), kMagic);
+}
 
 __device__ __forceinline__ void atomic_absmax(unsigned* addr, float v) {
   // non-negative floats order like their bit patterns

@@ -1,0 +1,313 @@
+// Hadamard stage of the Winograd-aware layer as t*t independent int8 GEMMs over
+// channels with int32 accumulation (paper: Sections 1 and 5.3, "element-wise
+// GEMM stage"):   M[xi][tau][k] = sum_c V_q[xi][tau][c] * U_q[xi][k][c]
+// followed by the quantizer of the Hadamard output (paper: Fig. 2).
+//
+//   k_gemm_tc   : persistent, warp-specialised tcgen05 kernel.  int8 operands are
+//                 staged in shared memory by TMA (128-byte swizzle), MMAs of
+//                 kind::i8 accumulate in int32 in tensor memory, two accumulator
+//                 buffers let the epilogue of one block overlap the MMAs of the
+//                 next.
+//   k_gemm_dp4a : the same contraction with 4-way integer dot products on the
+//                 ALUs; fallback for channel counts the TMA path cannot take.
+#include "wino_launch.h"
+#include "wino_ptx.cuh"
+
+namespace wino {
+
+// ---------------------------------------------------------------------------
+// ALU fallback.  Thread = (xi, tau, 4 consecutive k).
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(128)
+k_gemm_dp4a(const __grid_constant__ Params p, const int8_t* __restrict__ Vq,
+            const int8_t* __restrict__ Uq, void* __restrict__ out, int out_mode,
+            unsigned* __restrict__ absmaxM) {
+  const int C4 = p.C >> 2, K4 = p.K >> 2;
+  const int xi = blockIdx.z;
+  const long idx = blockIdx.x * (long)blockDim.x + threadIdx.x;
+  float vmax = 0.0f;
+  griddep_launch();
+  griddep_wait();
+  if (idx < (long)p.T * K4) {
+    const int k4 = (int)(idx % K4);
+    const int tau = (int)(idx / K4);
+    const int* v = reinterpret_cast<const int*>(Vq) + ((long)xi * p.T + tau) * C4;
+    const int* u = reinterpret_cast<const int*>(Uq) + ((long)xi * p.K + k4 * 4) * C4;
+    int acc[4] = {0, 0, 0, 0};
+    for (int c4 = 0; c4 < C4; ++c4) {
+      const int vv = __ldg(v + c4);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[j] = __dp4a(vv, __ldg(u + (long)j * C4 + c4), acc[j]);
+    }
+    const long o = ((long)xi * p.T + tau) * p.K + k4 * 4;
+    if (out_mode == kOutI32) {
+      *reinterpret_cast<int4*>(reinterpret_cast<int*>(out) + o) =
+          make_int4(acc[0], acc[1], acc[2], acc[3]);
+    } else {
+      uint32_t wv = 0;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        float r = quant_magic(__int2float_rn(acc[j]), p.mult_M, p.lo_M, p.hi_M);
+        wv |= (__float_as_uint(r) & 0xFFu) << (8 * j);
+      }
+      *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(out) + o) = wv;
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) vmax = fmaxf(vmax, fabsf(__int2float_rn(acc[j])));
+  }
+  if (absmaxM != nullptr) atomic_absmax(absmaxM, vmax);
+}
+
+int launch_gemm_dp4a(const Params& p, const LaunchOpt& o, const int8_t* Vq, const int8_t* Uq,
+                     void* out, int out_mode, unsigned* absmaxM, cudaStream_t st) {
+  const long total = (long)p.T * (p.K / 4);
+  dim3 grid((unsigned)((total + 127) / 128), 1, (unsigned)(p.t * p.t));
+  return launch_kernel(k_gemm_dp4a, grid, dim3(128), 0, st, o.pdl, p, Vq, Uq, out, out_mode,
+                       absmaxM);
+}
+
+// ---------------------------------------------------------------------------
+// tcgen05 GEMM.  Work item = one 128 (tau) x BN (k) block of one xi; CTAs walk
+// the item list with stride gridDim.x (m-block fastest, so CTAs running
+// together share the same U_q tile in L2).
+//   warp 0   : TMA producer (one lane)
+//   warp 1   : tensor-memory owner; one lane issues the MMAs
+//   warps 2-17: epilogue.  Warp w reads TMEM lanes 32*(w%4) .. +31 (its hardware
+//              quadrant) and every fourth 32-column chunk, by (w-2)/4, two chunks
+//              in flight at a time.
+// A stage holds 128 channels: A tile 128 x 128 B, B tile BN x 128 B; one MMA
+// consumes 32 channels.
+// ---------------------------------------------------------------------------
+struct GemmTcArgs {
+  int BN;          // multiple of 16, <= 256
+  int stages;
+  int tmem_cols;   // power of two >= 32, >= 2 * acc_stride
+  int acc_stride;  // columns between the two accumulator buffers
+  int out_mode;
+  int n_mblk, n_nblk, n_items;
+};
+
+constexpr int kEpiWarps = 16;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
+
+template <bool SMALL>
+__device__ __forceinline__ float acc_to_float(uint32_t v) {
+  if constexpr (SMALL) return small_int_to_float((int)v);
+  else return __int2float_rn((int)v);
+}
+
+template <bool SMALL>
+__device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (&r)[32], int k0,
+                                               long o, int out_mode, void* out, bool want_max,
+                                               float& vmax) {
+  if (want_max) {
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+      if (k0 + j < p.K) vmax = fmaxf(vmax, fabsf(__int2float_rn((int)r[j])));
+  }
+  if (out_mode == kOutI32) {
+    int4* dst = reinterpret_cast<int4*>(reinterpret_cast<int*>(out) + o);
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+      if (k0 + q * 4 < p.K)
+        dst[q] = make_int4((int)r[4 * q], (int)r[4 * q + 1], (int)r[4 * q + 2], (int)r[4 * q + 3]);
+  } else {
+    uint32_t w[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+      const float f0 = quant_magic(acc_to_float<SMALL>(r[4 * q + 0]), p.mult_M, p.lo_M, p.hi_M);
+      const float f1 = quant_magic(acc_to_float<SMALL>(r[4 * q + 1]), p.mult_M, p.lo_M, p.hi_M);
+      const float f2 = quant_magic(acc_to_float<SMALL>(r[4 * q + 2]), p.mult_M, p.lo_M, p.hi_M);
+      const float f3 = quant_magic(acc_to_float<SMALL>(r[4 * q + 3]), p.mult_M, p.lo_M, p.hi_M);
+      const uint32_t lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x0040u);
+      const uint32_t hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x0040u);
+      w[q] = __byte_perm(lo, hi, 0x5410u);
+    }
+    uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(out) + o);
+    if (k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    if (k0 + 16 < p.K) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+  }
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV,
+          const __grid_constant__ CUtensorMap mapU, const GemmTcArgs a, void* __restrict__ out,
+          unsigned* __restrict__ absmaxM, int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  // tiles need 1024-byte alignment for the 128-byte swizzle
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t a_bytes = kBM * kStageK, b_bytes = (uint32_t)a.BN * kStageK;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+  const uint32_t bars = base + (uint32_t)a.stages * stage_bytes;
+  const uint32_t bar_full = bars;                           // stages x 8 B
+  const uint32_t bar_empty = bar_full + 8u * a.stages;      // stages x 8 B
+  const uint32_t bar_acc_full = bar_empty + 8u * a.stages;  // 2 x 8 B
+  const uint32_t bar_acc_empty = bar_acc_full + 16u;        // 2 x 8 B
+  const uint32_t tmem_slot = bar_acc_empty + 16u;
+  const uint32_t abort_slot = tmem_slot + 4u;
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
+  volatile uint32_t* abort_p = reinterpret_cast<volatile uint32_t*>(gen + (abort_slot - base));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int KB = (p.C + kStageK - 1) / kStageK;
+  const int per_xi = a.n_mblk * a.n_nblk;
+
+  griddep_launch();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < a.stages; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_acc_full + 8u * b, 1);
+      mbar_init(bar_acc_empty + 8u * b, kEpiWarps);
+    }
+    *abort_p = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, (uint32_t)a.tmem_cols);
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_p;
+  griddep_wait();   // everything below reads or writes buffers other kernels touch
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int s = 0; uint32_t ph = 0;
+      for (int it = blockIdx.x; it < a.n_items; it += gridDim.x) {
+        const int xi = it / per_xi, rem = it - xi * per_xi;
+        const int nb = rem / a.n_mblk, mb = rem - nb * a.n_mblk;
+        bool ok = true;
+        for (int kb = 0; kb < KB; ++kb) {
+          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
+          const uint32_t sa = base + (uint32_t)s * stage_bytes;
+          mbar_expect_tx(bar_full + 8u * s, stage_bytes);
+          tma_load_3d(sa, &mapV, bar_full + 8u * s, kb * kStageK, mb * kBM, xi);
+          tma_load_3d(sa + a_bytes, &mapU, bar_full + 8u * s, kb * kStageK, nb * a.BN, xi);
+          if (++s == a.stages) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) { *abort_p = 1u; break; }
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {
+      const uint32_t idesc = make_idesc_i8(kBM, a.BN);
+      int s = 0; uint32_t ph = 0;
+      int li = 0;
+      for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
+        const int buf = li & 1;
+        const uint32_t aph = (uint32_t)(li >> 1) & 1u;
+        bool ok = mbar_wait(bar_acc_empty + 8u * buf, aph ^ 1u, abort_p);
+        tc_fence_after();
+        const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride);
+        for (int kb = 0; kb < KB && ok; ++kb) {
+          if (!mbar_wait(bar_full + 8u * s, ph, abort_p)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t sa = base + (uint32_t)s * stage_bytes;
+          const uint64_t da = make_desc_sw128(sa), db = make_desc_sw128(sa + a_bytes);
+          const int remc = p.C - kb * kStageK;
+          const int ksteps = remc >= kStageK ? 4 : (remc + 31) / 32;
+          for (int k = 0; k < ksteps; ++k)
+            mma_i8(tacc, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
+                   (kb | k) != 0 ? 1u : 0u);
+          mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
+          if (++s == a.stages) { s = 0; ph ^= 1u; }
+        }
+        if (!ok) { *abort_p = 1u; break; }
+        mma_commit(bar_acc_full + 8u * buf);  // accumulator complete
+      }
+    }
+  } else {
+    // epilogue warps
+    const int quad = warp & 3;
+    const int sub = (warp - 2) >> 2;
+    const bool small = p.C <= 260;   // |M| <= 127^2 * C < 2^22
+    const bool want_max = absmaxM != nullptr;
+    float vmax = 0.0f;
+    int li = 0;
+    for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
+      const int xi = it / per_xi, rem = it - xi * per_xi;
+      const int nb = rem / a.n_mblk, mb = rem - nb * a.n_mblk;
+      const int buf = li & 1;
+      const uint32_t aph = (uint32_t)(li >> 1) & 1u;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8u * buf, aph, abort_p))) {
+        *abort_p = 1u;
+        break;
+      }
+      tc_fence_after();
+      const int tau = mb * kBM + quad * 32 + lane;
+      const bool row_ok = tau < p.T;
+      const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride) + ((uint32_t)(quad * 32) << 16);
+      for (int col = sub * 32; col < a.BN; col += 256) {
+        // two chunks in flight: col and col + 128
+        const bool two = col + 128 < a.BN;
+        uint32_t r0[32], r1[32];
+        tmem_ld32(tacc + (uint32_t)col, r0);
+        if (two) tmem_ld32(tacc + (uint32_t)(col + 128), r1);
+        tmem_ld_wait();
+        if (!row_ok) continue;
+        const int k0 = nb * a.BN + col;
+        const long o = ((long)xi * p.T + tau) * p.K + k0;
+        if (small) {
+          epilogue_chunk<true>(p, r0, k0, o, a.out_mode, out, want_max, vmax);
+          if (two) epilogue_chunk<true>(p, r1, k0 + 128, o + 128, a.out_mode, out, want_max, vmax);
+        } else {
+          epilogue_chunk<false>(p, r0, k0, o, a.out_mode, out, want_max, vmax);
+          if (two) epilogue_chunk<false>(p, r1, k0 + 128, o + 128, a.out_mode, out, want_max, vmax);
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty + 8u * buf);
+    }
+    if (want_max) atomic_absmax(absmaxM, vmax);
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_p != 0u && threadIdx.x == 0) atomicExch(status, -6);  // WINO_ERR_TIMEOUT
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+  }
+}
+
+TcGeom tc_geometry(const Params& p, int num_sms) {
+  TcGeom g;
+  g.BN = p.K >= 256 ? 256 : (p.K + 15) / 16 * 16;
+  const size_t per_stage = (size_t)kBM * kStageK + (size_t)g.BN * kStageK;
+  g.stages = (int)((196 * 1024) / per_stage);
+  if (g.stages > 8) g.stages = 8;
+  if (g.stages < 1) g.stages = 1;
+  int acc_stride = 32;
+  while (acc_stride < g.BN) acc_stride *= 2;
+  g.tmem_cols = 2 * acc_stride;
+  g.smem = 1024 + g.stages * per_stage + 16 * g.stages + 64;
+  const int items = (p.t * p.t) * ((p.T + kBM - 1) / kBM) * ((p.K + g.BN - 1) / g.BN);
+  g.grid = items < num_sms ? items : num_sms;
+  return g;
+}
+
+int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,
+                   const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
+                   int* status, cudaStream_t st) {
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
+        cudaSuccess)
+      return -5;
+    attr_set = true;
+  }
+  GemmTcArgs a;
+  a.BN = g.BN; a.stages = g.stages; a.tmem_cols = g.tmem_cols; a.acc_stride = g.tmem_cols / 2;
+  a.out_mode = out_mode;
+  a.n_mblk = (p.T + kBM - 1) / kBM;
+  a.n_nblk = (p.K + g.BN - 1) / g.BN;
+  a.n_items = p.t * p.t * a.n_mblk * a.n_nblk;
+  return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,
+                       mapV, mapU, a, out, absmaxM, status);
+}
+
+}  // namespace wino

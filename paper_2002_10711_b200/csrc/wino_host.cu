@@ -10,10 +10,7 @@
 #include <cuda_runtime.h>
 
 #include "wino.h"
-#include "wino_common.cuh"
-#include "wino_gemm.cuh"
-#include "wino_smallc.cuh"
-#include "wino_transforms.cuh"
+#include "wino_launch.h"
 
 using namespace wino;
 
@@ -22,6 +19,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+// Small round-robin memo of encoded tensor maps keyed by the buffer address.
+struct MapCache {
+  static constexpr int kN = 32;
+  const void* key[kN];
+  CUtensorMap map[kN];
+  int next;
+  const CUtensorMap* find(const void* k) const {
+    for (int i = 0; i < kN; ++i)
+      if (key[i] == k) return &map[i];
+    return nullptr;
+  }
+  CUtensorMap* slot(const void* k) {
+    const int i = next;
+    next = (next + 1) % kN;
+    key[i] = k;
+    return &map[i];
+  }
+};
+
 struct wino_plan {
   wino_desc_t d;
   Params p;
@@ -29,11 +45,14 @@ struct wino_plan {
   bool std_mats;        // BT and AT equal the built-in Cook-Toom matrices bit for bit
   int path;
   int* status_dev;      // device status word (may be null when no GPU is present)
-  bool tc_attr_set;
+  int num_sms;
+  bool pdl;             // programmatic dependent launch between the stages
   // memo of the last encoded tensor maps
   mutable const void* map_vq_ptr;
   mutable const void* map_uq_ptr;
   mutable CUtensorMap mapV, mapU;
+  // maps of the TMA-staged transform kernels, keyed by buffer address
+  mutable MapCache cache_x, cache_vst, cache_mld, cache_y;
   // last forward call, for wino_debug_dump_stage
   mutable const int8_t* last_uq;
   mutable void* last_ws;
@@ -83,7 +102,8 @@ bool is_std(const float* BT, const float* AT) {
 bool path_supported(const wino_plan_t* pl, int path) {
   const int C = pl->d.C, K = pl->d.K;
   switch (path) {
-    case WINO_PATH_STAGED_TC: return C % 16 == 0 && K % 16 == 0;
+    case WINO_PATH_STAGED_TC:
+    case WINO_PATH_STAGED_TC_PTR: return C % 16 == 0 && K % 16 == 0;
     case WINO_PATH_STAGED_DP4A: return C % 4 == 0 && K % 4 == 0;
     case WINO_PATH_SMALLC: return C % 4 == 0 && K % 4 == 0 && C <= 32 && K <= 32;
     default: return false;
@@ -94,93 +114,87 @@ size_t vq_bytes(const wino_plan_t* pl) { return (size_t)pl->p.t * pl->p.t * pl->
 size_t m_elems(const wino_plan_t* pl) { return (size_t)pl->p.t * pl->p.t * pl->p.T * pl->p.K; }
 size_t mbuf_bytes(const wino_plan_t* pl) { return m_elems(pl) * (pl->p.qM_enabled ? 1 : 4); }
 
-int check_launch(const wino_plan_t* pl) {
-  pl->launches++;
-  return cudaGetLastError() == cudaSuccess ? WINO_OK : WINO_ERR_CUDA;
+LaunchOpt opt_of(const wino_plan_t* pl, bool pdl) {
+  LaunchOpt o;
+  o.std_mats = pl->std_mats;
+  o.pdl = pdl;
+  return o;
 }
 
-// --- launches -------------------------------------------------------------
-template <int M>
-int launch_weight(const wino_plan_t* pl, const int8_t* w, int8_t* Uq, unsigned* absmax,
-                  cudaStream_t st) {
-  const long total = (long)pl->p.K * (pl->p.C / 4);
-  const int grid = (int)((total + 127) / 128);
-  k_weight_transform<M><<<grid, 128, 0, st>>>(pl->p, w, Uq, absmax);
-  return check_launch(pl);
-}
-
-template <int M>
-int launch_input(const wino_plan_t* pl, const int8_t* x, int8_t* Vq, unsigned* absmax,
-                 cudaStream_t st) {
-  const long total = (long)pl->p.T * (pl->p.C / 4);
-  const int grid = (int)((total + 127) / 128);
-  if (pl->std_mats)
-    k_input_transform<M, true><<<grid, 128, 0, st>>>(pl->p, x, Vq, absmax);
-  else
-    k_input_transform<M, false><<<grid, 128, 0, st>>>(pl->p, x, Vq, absmax);
-  return check_launch(pl);
-}
-
-template <int M>
-int launch_output(const wino_plan_t* pl, const void* mbuf, const float* bias, void* y,
-                  unsigned* absmax2, cudaStream_t st) {
-  const long total = (long)pl->p.T * (pl->p.K / 4);
-  const int grid = (int)((total + 127) / 128);
-  const bool qm = pl->p.qM_enabled != 0;
-  if (pl->std_mats) {
-    if (qm) k_output_transform<M, true, true><<<grid, 128, 0, st>>>(pl->p, mbuf, bias, y, pl->s_Y, absmax2);
-    else k_output_transform<M, true, false><<<grid, 128, 0, st>>>(pl->p, mbuf, bias, y, pl->s_Y, absmax2);
-  } else {
-    if (qm) k_output_transform<M, false, true><<<grid, 128, 0, st>>>(pl->p, mbuf, bias, y, pl->s_Y, absmax2);
-    else k_output_transform<M, false, false><<<grid, 128, 0, st>>>(pl->p, mbuf, bias, y, pl->s_Y, absmax2);
-  }
-  return check_launch(pl);
-}
-
-#define DISPATCH_M(pl, call)                         \
-  ((pl)->p.m == 2 ? call<2> : (pl)->p.m == 4 ? call<4> : call<6>)
-
-int encode_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t mats,
-               uint32_t box_rows) {
+int encode_tiled(CUtensorMap* map, const void* base, int rank, const uint64_t* dims,
+                 const uint32_t* box, CUtensorMapSwizzle swz) {
   EncodeTiledFn fn = get_encode_fn();
   if (fn == nullptr) return WINO_ERR_CUDA;
-  cuuint64_t dims[3] = {inner, rows, mats};
-  cuuint64_t strides[2] = {inner, inner * rows};  // bytes (int8 elements)
-  cuuint32_t box[3] = {(cuuint32_t)kStageK, box_rows, 1};
-  cuuint32_t estr[3] = {1, 1, 1};
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides,
-                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+  cuuint64_t d[4], strides[3];
+  cuuint32_t b[4], estr[4] = {1, 1, 1, 1};
+  uint64_t stride = 1;
+  for (int i = 0; i < rank; ++i) {
+    d[i] = dims[i];
+    b[i] = box[i];
+    stride *= dims[i];
+    if (i < rank - 1) strides[i] = stride;  // bytes: int8 elements
+  }
+  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d,
+                  strides, b, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? WINO_OK : WINO_ERR_CUDA;
 }
 
-struct TcGeom { int BN, stages, tmem_cols; size_t smem; };
+int encode_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows, uint64_t mats,
+               uint32_t box_rows) {
+  const uint64_t dims[3] = {inner, rows, mats};
+  const uint32_t box[3] = {(uint32_t)kStageK, box_rows, 1};
+  return encode_tiled(map, base, 3, dims, box, CU_TENSOR_MAP_SWIZZLE_128B);
+}
 
-TcGeom tc_geom(const wino_plan_t* pl) {
-  TcGeom g;
-  const int K = pl->p.K;
-  g.BN = K >= 256 ? 256 : (int)round_up((size_t)K, 16);
-  const int KB = (pl->p.C + kStageK - 1) / kStageK;
-  g.stages = KB < 4 ? KB : 4;
-  const size_t per_stage = (size_t)kBM * kStageK + (size_t)g.BN * kStageK;
-  while (g.stages > 1 && g.stages * per_stage > 200 * 1024) --g.stages;
-  g.tmem_cols = 32;
-  while (g.tmem_cols < g.BN) g.tmem_cols *= 2;
-  g.smem = 1024 + g.stages * per_stage + 16 * g.stages + 64;
-  return g;
+// Tensor maps of the TMA-staged transform kernels (no swizzle).
+const CUtensorMap* map_x(const wino_plan_t* pl, const void* x) {
+  if (const CUtensorMap* m = pl->cache_x.find(x)) return m;
+  const Params& p = pl->p;
+  const uint64_t dims[4] = {(uint64_t)p.C, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.N};
+  const uint32_t box[4] = {(uint32_t)tma_chunk(p.C), (uint32_t)p.t, (uint32_t)p.t, 1};
+  CUtensorMap* m = pl->cache_x.slot(x);
+  if (encode_tiled(m, x, 4, dims, box, CU_TENSOR_MAP_SWIZZLE_NONE) != WINO_OK) {
+    pl->cache_x.key[(pl->cache_x.next + MapCache::kN - 1) % MapCache::kN] = nullptr;
+    return nullptr;
+  }
+  return m;
+}
+const CUtensorMap* map_y(const wino_plan_t* pl, const void* y) {
+  if (const CUtensorMap* m = pl->cache_y.find(y)) return m;
+  const Params& p = pl->p;
+  const uint64_t dims[4] = {(uint64_t)p.K, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.N};
+  const uint32_t box[4] = {(uint32_t)tma_chunk(p.K), (uint32_t)p.m, (uint32_t)p.m, 1};
+  CUtensorMap* m = pl->cache_y.slot(y);
+  if (encode_tiled(m, y, 4, dims, box, CU_TENSOR_MAP_SWIZZLE_NONE) != WINO_OK) {
+    pl->cache_y.key[(pl->cache_y.next + MapCache::kN - 1) % MapCache::kN] = nullptr;
+    return nullptr;
+  }
+  return m;
+}
+// V_q (store side) and m_q (load side): [t*t][T][channels], box {chunk, G, t*t}
+const CUtensorMap* map_stage(const wino_plan_t* pl, MapCache& cache, const void* buf, int channels) {
+  if (const CUtensorMap* m = cache.find(buf)) return m;
+  const Params& p = pl->p;
+  const int chunk = tma_chunk(channels);
+  const uint64_t dims[3] = {(uint64_t)channels, (uint64_t)p.T, (uint64_t)(p.t * p.t)};
+  const uint32_t box[3] = {(uint32_t)chunk, (uint32_t)tma_group(chunk), (uint32_t)(p.t * p.t)};
+  CUtensorMap* m = cache.slot(buf);
+  if (encode_tiled(m, buf, 3, dims, box, CU_TENSOR_MAP_SWIZZLE_NONE) != WINO_OK) {
+    cache.key[(cache.next + MapCache::kN - 1) % MapCache::kN] = nullptr;
+    return nullptr;
+  }
+  return m;
 }
 
 int launch_gemm(const wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void* out, int out_mode,
-                unsigned* absmaxM, cudaStream_t st) {
+                unsigned* absmaxM, bool pdl, cudaStream_t st) {
   const Params& p = pl->p;
   const int t2 = p.t * p.t;
-  if (pl->path == WINO_PATH_STAGED_DP4A) {
-    const long total = (long)p.T * (p.K / 4);
-    dim3 grid((unsigned)((total + 127) / 128), 1, (unsigned)t2);
-    k_gemm_dp4a<<<grid, 128, 0, st>>>(p, Vq, Uq, out, out_mode, absmaxM);
-    return check_launch(pl);
-  }
-  TcGeom g = tc_geom(pl);
+  pl->launches++;
+  if (pl->path == WINO_PATH_STAGED_DP4A)
+    return launch_gemm_dp4a(p, opt_of(pl, pdl), Vq, Uq, out, out_mode, absmaxM, st);
+  const TcGeom g = tc_geometry(p, pl->num_sms);
   if (pl->map_vq_ptr != Vq) {
     int rc = encode_map(&pl->mapV, Vq, (uint64_t)p.C, (uint64_t)p.T, (uint64_t)t2, kBM);
     if (rc != WINO_OK) return rc;
@@ -191,33 +205,24 @@ int launch_gemm(const wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void*
     if (rc != WINO_OK) return rc;
     pl->map_uq_ptr = Uq;
   }
-  if (!pl->tc_attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024) !=
-        cudaSuccess)
-      return WINO_ERR_CUDA;
-    const_cast<wino_plan_t*>(pl)->tc_attr_set = true;
-  }
-  GemmTcArgs a;
-  a.BN = g.BN; a.stages = g.stages; a.tmem_cols = g.tmem_cols; a.out_mode = out_mode;
-  dim3 grid((unsigned)((p.T + kBM - 1) / kBM), (unsigned)((p.K + g.BN - 1) / g.BN), (unsigned)t2);
-  k_gemm_tc<<<grid, 128, g.smem, st>>>(p, pl->mapV, pl->mapU, a, out, absmaxM, pl->status_dev);
-  return check_launch(pl);
+  return launch_gemm_tc(p, opt_of(pl, pdl), g, pl->mapV, pl->mapU, out, out_mode, absmaxM,
+                        pl->status_dev, st);
 }
 
 int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias, void* y,
                  void* ws, unsigned* absmax4, cudaStream_t st) {
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
   const bool calib = absmax4 != nullptr;
+  const bool pdl = pl->pdl && !calib;
   if (pl->path == WINO_PATH_SMALLC && !calib) {
-    int rc = launch_smallc(pl->p, pl->std_mats, x, Uq, bias, y, pl->s_Y, st);
     pl->launches++;
-    return rc == 0 && cudaGetLastError() == cudaSuccess ? WINO_OK : WINO_ERR_CUDA;
+    return launch_smallc(pl->p, opt_of(pl, pdl), x, Uq, bias, y, pl->s_Y, st);
   }
   if (ws == nullptr) return WINO_ERR_WORKSPACE;
   if (!aligned16(ws)) return WINO_ERR_ALIGNMENT;
   int8_t* Vq = reinterpret_cast<int8_t*>(ws);
   void* mbuf = reinterpret_cast<uint8_t*>(ws) + round_up(vq_bytes(pl), 1024);
-  // calibration on a small-channel plan uses the dp4a kernels for the middle stage
+  // calibration on a small-channel plan uses the dp4a kernel for the middle stage
   wino_plan_t tmp_holder;
   const wino_plan_t* run = pl;
   if (pl->path == WINO_PATH_SMALLC) {
@@ -227,15 +232,38 @@ int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const
   }
   const bool ev = pl->stage_ev_on;
   if (ev) cudaEventRecord(pl->stage_ev[0], st);
-  int rc = DISPATCH_M(pl, launch_input)(pl, x, Vq, calib ? absmax4 + 0 : nullptr, st);
+  pl->launches++;
+  const bool tma_ok = pl->path == WINO_PATH_STAGED_TC && !calib;
+  int rc;
+  if (tma_ok && pl->p.z_x == 0 && tma_chunk(pl->p.C) != 0) {
+    const CUtensorMap* mx = map_x(pl, x);
+    const CUtensorMap* mv = map_stage(pl, pl->cache_vst, Vq, pl->p.C);
+    if (mx == nullptr || mv == nullptr) return WINO_ERR_CUDA;
+    rc = launch_input_transform_tma(pl->p, opt_of(pl, pdl && !ev), *mx, *mv, pl->status_dev, st);
+  } else {
+    rc = launch_input_transform(pl->p, opt_of(pl, pdl && !ev), x, Vq, calib ? absmax4 + 0 : nullptr,
+                                st);
+  }
   if (rc != WINO_OK) return rc;
   if (ev) cudaEventRecord(pl->stage_ev[1], st);
   rc = launch_gemm(run, Vq, Uq, mbuf, pl->p.qM_enabled ? kOutMq : kOutI32,
-                   calib ? absmax4 + 1 : nullptr, st);
-  if (run != pl) pl->launches++;
+                   calib ? absmax4 + 1 : nullptr, pdl && !ev, st);
+  if (run != pl) {
+    pl->launches++;
+  }
   if (rc != WINO_OK) return rc;
   if (ev) cudaEventRecord(pl->stage_ev[2], st);
-  rc = DISPATCH_M(pl, launch_output)(pl, mbuf, bias, y, calib ? absmax4 + 2 : nullptr, st);
+  pl->launches++;
+  if (tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
+    const CUtensorMap* mm = map_stage(pl, pl->cache_mld, mbuf, pl->p.K);
+    const CUtensorMap* my = map_y(pl, y);
+    if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
+    rc = launch_output_transform_tma(pl->p, opt_of(pl, pdl && !ev), *mm, *my, bias, pl->s_Y,
+                                     pl->status_dev, st);
+  } else {
+    rc = launch_output_transform(pl->p, opt_of(pl, pdl && !ev), pl->s_Y, mbuf, bias, y,
+                                 calib ? absmax4 + 2 : nullptr, st);
+  }
   if (rc != WINO_OK) return rc;
   if (ev) cudaEventRecord(pl->stage_ev[3], st);
   pl->last_uq = Uq;
@@ -308,8 +336,14 @@ int wino_plan(const wino_desc_t* desc, wino_plan_t** out) {
   else if (path_supported(pl, WINO_PATH_STAGED_TC)) pl->path = WINO_PATH_STAGED_TC;
   else if (path_supported(pl, WINO_PATH_STAGED_DP4A)) pl->path = WINO_PATH_STAGED_DP4A;
   else { delete pl; return WINO_ERR_UNSUPPORTED; }
+  pl->num_sms = 148;
+  pl->pdl = true;
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess &&
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+      pl->num_sms = sms;
     if (cudaMalloc(&pl->status_dev, 256) == cudaSuccess) {
       cudaMemset(pl->status_dev, 0, 256);
     } else {
@@ -335,7 +369,7 @@ int wino_plan_path(const wino_plan_t* pl) { return pl ? pl->path : WINO_ERR_INVA
 
 int wino_plan_force_path(wino_plan_t* pl, int path) {
   if (pl == nullptr) return WINO_ERR_INVALID;
-  if (path < WINO_PATH_STAGED_TC || path > WINO_PATH_SMALLC) return WINO_ERR_INVALID;
+  if (path < WINO_PATH_STAGED_TC || path > WINO_PATH_STAGED_TC_PTR) return WINO_ERR_INVALID;
   if (!path_supported(pl, path)) return WINO_ERR_UNSUPPORTED;
   pl->path = path;
   return WINO_OK;
@@ -354,7 +388,8 @@ int wino_transform_weights(const wino_plan_t* pl, const int8_t* w, int8_t* Uq, u
   if (pl == nullptr || w == nullptr || Uq == nullptr) return WINO_ERR_INVALID;
   if (!aligned16(w) || !aligned16(Uq)) return WINO_ERR_ALIGNMENT;
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
-  return DISPATCH_M(pl, launch_weight)(pl, w, Uq, absmax, (cudaStream_t)stream);
+  pl->launches++;
+  return launch_weight_transform(pl->p, w, Uq, absmax, (cudaStream_t)stream);
 }
 
 int wino_conv_forward(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias,
@@ -405,11 +440,10 @@ int wino_debug_dump_stage(const wino_plan_t* pl, int stage, void* dst, size_t by
     wino_plan_t tmp = *pl;
     if (tmp.path == WINO_PATH_SMALLC) tmp.path = WINO_PATH_STAGED_DP4A;
     int rc = launch_gemm(&tmp, reinterpret_cast<const int8_t*>(ws), pl->last_uq, dst, kOutI32,
-                         nullptr, st);
+                         nullptr, false, st);
     pl->launches++;
     pl->map_vq_ptr = tmp.map_vq_ptr; pl->map_uq_ptr = tmp.map_uq_ptr;
     pl->mapV = tmp.mapV; pl->mapU = tmp.mapU;
-    const_cast<wino_plan_t*>(pl)->tc_attr_set = tmp.tc_attr_set;
     return rc;
   }
   return WINO_ERR_INVALID;

@@ -1,0 +1,65 @@
+// Internal interface between the host planner (wino_host.cu) and the kernel
+// translation units.  Every function enqueues work on `st` and returns 0 or a
+// negative WINO_ERR_* code; none allocates or synchronizes.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include "wino_common.cuh"
+
+namespace wino {
+
+// Launch options shared by all kernels.
+struct LaunchOpt {
+  bool std_mats = false;      // B^T and A^T are the built-in Cook-Toom matrices
+  bool pdl = false;           // programmatic dependent launch on the stream
+};
+
+int launch_weight_transform(const Params& p, const int8_t* w, int8_t* Uq, unsigned* absmax,
+                            cudaStream_t st);
+int launch_input_transform(const Params& p, const LaunchOpt& o, const int8_t* x, int8_t* Vq,
+                           unsigned* absmax, cudaStream_t st);
+int launch_output_transform(const Params& p, const LaunchOpt& o, float s_Y, const void* mbuf,
+                            const float* bias, void* y, unsigned* absmax2, cudaStream_t st);
+int launch_gemm_dp4a(const Params& p, const LaunchOpt& o, const int8_t* Vq, const int8_t* Uq,
+                     void* out, int out_mode, unsigned* absmaxM, cudaStream_t st);
+
+// TMA-staged transform kernels (input needs z_x == 0 and C % 64 == 0; output needs
+// Q_M on, int8 output and K % 64 == 0).  Channel chunk per block:
+inline int tma_chunk(int channels) {
+  return channels % 256 == 0 ? 256 : channels % 128 == 0 ? 128 : channels % 64 == 0 ? 64 : 0;
+}
+inline int tma_group(int chunk) { return chunk == 256 ? 1 : chunk == 128 ? 2 : 4; }
+int launch_input_transform_tma(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX,
+                               const CUtensorMap& mapV, int* status, cudaStream_t st);
+int launch_output_transform_tma(const Params& p, const LaunchOpt& o, const CUtensorMap& mapM,
+                                const CUtensorMap& mapY, const float* bias, float s_Y, int* status,
+                                cudaStream_t st);
+
+struct TcGeom { int BN, stages, tmem_cols, grid; size_t smem; };
+TcGeom tc_geometry(const Params& p, int num_sms);
+int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,
+                   const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
+                   int* status, cudaStream_t st);
+int launch_smallc(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
+                  const float* bias, void* y, float s_Y, cudaStream_t st);
+
+enum { kOutMq = 0, kOutI32 = 1 };
+constexpr int kBM = 128;      // tiles per GEMM block (MMA M)
+constexpr int kStageK = 128;  // channels (bytes) per shared-memory stage
+
+// Generic launcher: plain <<<>>> or cudaLaunchKernelEx with the programmatic
+// stream serialization attribute (the kernel then calls griddep_wait()).
+template <typename... KArgs, typename... Args>
+int launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                  bool pdl, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = pdl ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) == cudaSuccess ? 0 : -5;
+}
+
+}  // namespace wino

@@ -10,8 +10,7 @@
 //     products against U_q held in shared memory;
 //   - lane = k for Q_M, the output transform A^T m A, bias and Q_Y.
 // Nothing but x, U_q and y touches global memory.
-#pragma once
-#include "wino_common.cuh"
+#include "wino_launch.h"
 
 namespace wino {
 
@@ -24,6 +23,8 @@ k_smallc(const __grid_constant__ Params p, const int8_t* __restrict__ x,
   using MT = Mat<M, STD>;
   extern __shared__ uint32_t sU[];  // [T2][C4][K]: word L of filter (xi, k)
   const int C4 = p.C >> 2, K = p.K;
+  griddep_launch();
+  griddep_wait();
   {
     const uint32_t* U32 = reinterpret_cast<const uint32_t*>(Uq);
     const int per_xi = K * C4;
@@ -122,30 +123,36 @@ k_smallc(const __grid_constant__ Params p, const int8_t* __restrict__ x,
   }
 }
 
-template <int M>
-int launch_smallc_m(const Params& p, bool std_mats, const int8_t* x, const int8_t* Uq,
-                    const float* bias, void* y, float s_Y, cudaStream_t st) {
+namespace {
+template <int M, bool STD>
+int smallc_launch(const Params& p, bool pdl, const int8_t* x, const int8_t* Uq, const float* bias,
+                  void* y, float s_Y, cudaStream_t st) {
   constexpr int T2 = (M + 2) * (M + 2);
   const size_t smem = (size_t)T2 * (p.C / 4) * p.K * 4;
+  static bool attr_set = false;   // one flag per instantiation
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k_smallc<M, STD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             64 * 32 * 8 * 4) != cudaSuccess) return -5;
+    attr_set = true;
+  }
   int blocks = (p.T + 3) / 4;
   if (blocks > 148 * 8) blocks = 148 * 8;
-  if (std_mats) {
-    if (cudaFuncSetAttribute(k_smallc<M, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess) return -1;
-    k_smallc<M, true><<<blocks, 128, smem, st>>>(p, x, Uq, bias, y, s_Y);
-  } else {
-    if (cudaFuncSetAttribute(k_smallc<M, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess) return -1;
-    k_smallc<M, false><<<blocks, 128, smem, st>>>(p, x, Uq, bias, y, s_Y);
-  }
-  return 0;
+  return launch_kernel(k_smallc<M, STD>, dim3((unsigned)blocks), dim3(128), smem, st, pdl, p, x, Uq,
+                       bias, y, s_Y);
 }
+template <int M>
+int smallc_m(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
+             const float* bias, void* y, float s_Y, cudaStream_t st) {
+  return o.std_mats ? smallc_launch<M, true>(p, o.pdl, x, Uq, bias, y, s_Y, st)
+                    : smallc_launch<M, false>(p, o.pdl, x, Uq, bias, y, s_Y, st);
+}
+}  // namespace
 
-inline int launch_smallc(const Params& p, bool std_mats, const int8_t* x, const int8_t* Uq,
-                         const float* bias, void* y, float s_Y, cudaStream_t st) {
-  return p.m == 2 ? launch_smallc_m<2>(p, std_mats, x, Uq, bias, y, s_Y, st)
-       : p.m == 4 ? launch_smallc_m<4>(p, std_mats, x, Uq, bias, y, s_Y, st)
-                  : launch_smallc_m<6>(p, std_mats, x, Uq, bias, y, s_Y, st);
+int launch_smallc(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
+                  const float* bias, void* y, float s_Y, cudaStream_t st) {
+  return p.m == 2 ? smallc_m<2>(p, o, x, Uq, bias, y, s_Y, st)
+       : p.m == 4 ? smallc_m<4>(p, o, x, Uq, bias, y, s_Y, st)
+                  : smallc_m<6>(p, o, x, Uq, bias, y, s_Y, st);
 }
 
 }  // namespace wino

@@ -1,0 +1,256 @@
+// TMA-staged variants of the input and output transform kernels (paper: Eq. 1,
+// Fig. 2, stages 1 and 4).  A block owns G consecutive tiles x CC channels:
+//   - the (m+2)x(m+2)xCC input patches (or the t*t x G x CC block of m_q) arrive
+//     in shared memory by TMA; for the input, coordinates may start at -1 and
+//     run past the image: the hardware fills those bytes with zero, which is
+//     the padding (valid when the input zero point is 0);
+//   - every thread transforms four channels from registers, reading and writing
+//     shared memory at compile-time offsets;
+//   - the result leaves by one TMA store (rows past the last tile, or pixels past
+//     the image edge, are clipped by the hardware).
+// Compared with the pointer-based kernels this removes nearly all integer
+// address arithmetic, which was a third of their instructions.
+#pragma once
+#include "wino_ptx.cuh"
+
+namespace wino {
+
+template <int M, int MODE, int CC, int G>
+__global__ void __launch_bounds__((CC / 4) * G)
+k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
+                      const __grid_constant__ CUtensorMap mapV, int* __restrict__ status) {
+  constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / 4;
+  constexpr uint32_t kTileBytes = T2 * CC;
+  constexpr uint32_t kUnitBytes = G * kTileBytes;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+  const uint32_t s_in = base;                 // [G][T2][CC]
+  const uint32_t s_out = base + kUnitBytes;   // [T2][G][CC]
+  const uint32_t bar = s_out + kUnitBytes;
+  __shared__ uint32_t abort_flag;
+
+  const int cchunks = p.C / CC;
+  const int unit = blockIdx.x;
+  const int tau0 = (unit / cchunks) * G;
+  const int c0 = (unit % cchunks) * CC;
+  const int g = threadIdx.x / TPT, c4 = threadIdx.x % TPT;
+  const int ntile = min(G, p.T - tau0);
+
+  griddep_launch();
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  griddep_wait();
+  if (threadIdx.x == 0) {
+    mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
+    for (int i = 0; i < ntile; ++i) {
+      const int tau = tau0 + i;
+      const int tw = tau % p.TW;
+      const int th = (tau / p.TW) % p.TH;
+      const int n = tau / (p.TW * p.TH);
+      tma_load_4d(s_in + (uint32_t)i * kTileBytes, &mapX, bar, c0, tw * M - 1, th * M - 1, n);
+    }
+  }
+  const bool ok = __syncthreads_and(mbar_wait(bar, 0u, &abort_flag) ? 1 : 0) != 0;
+  if (!ok) {
+    if (threadIdx.x == 0) atomicExch(status, -6);  // WINO_ERR_TIMEOUT
+    return;
+  }
+  if (g < ntile) {
+    const uint32_t rd = s_in + (uint32_t)g * kTileBytes + 4u * (uint32_t)c4;
+    uint32_t wd[T2];
+#pragma unroll
+    for (int ab = 0; ab < T2; ++ab) wd[ab] = lds32(rd + (uint32_t)ab * CC) ^ 0x80808080u;
+    uint32_t out[T2];
+#pragma unroll
+    for (int i = 0; i < T2; ++i) out[i] = 0u;
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ++ch) {
+      const uint32_t sel_in = 0x7440u | (uint32_t)ch;
+      const uint32_t sel_out = insert_selector(ch);
+      float V[T2];
+      input_transform_2d<M, MODE>(p, [&](int l, float (&dcol)[T_]) {
+#pragma unroll
+        for (int a = 0; a < T_; ++a) dcol[a] = byte_to_float_sel(wd[a * T_ + l], sel_in, 8388736.0f);
+      }, V);
+#pragma unroll
+      for (int xi = 0; xi < T2; ++xi) {
+        const float r = quant_magic(V[xi], p.mult_V, p.lo_V, p.hi_V);
+        out[xi] = __byte_perm(out[xi], __float_as_uint(r), sel_out);
+      }
+    }
+    const uint32_t wr = s_out + ((uint32_t)g * CC + 4u * (uint32_t)c4);
+#pragma unroll
+    for (int xi = 0; xi < T2; ++xi) sts32(wr + (uint32_t)xi * (G * CC), out[xi]);
+  }
+  fence_async_smem();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    tma_store_3d(&mapV, s_out, c0, tau0, 0);
+    bulk_commit();
+    bulk_wait_all();
+  }
+}
+
+template <int M, int MODE, int KC, int G>
+__global__ void __launch_bounds__((KC / 4) * G)
+k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapM,
+                       const __grid_constant__ CUtensorMap mapY, const float* __restrict__ bias,
+                       float s_Y, int* __restrict__ status) {
+  constexpr int T_ = M + 2, T2 = T_ * T_, TPT = KC / 4;
+  constexpr uint32_t kInBytes = T2 * G * KC;          // [T2][G][KC]
+  constexpr uint32_t kTileOut = M * M * KC;           // [M][M][KC] per tile
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
+  const uint32_t s_in = base;
+  const uint32_t s_out = base + kInBytes;             // [G][M][M][KC]
+  const uint32_t bar = s_out + G * kTileOut;
+  __shared__ uint32_t abort_flag;
+
+  const int kchunks = p.K / KC;
+  const int unit = blockIdx.x;
+  const int tau0 = (unit / kchunks) * G;
+  const int k0 = (unit % kchunks) * KC;
+  const int g = threadIdx.x / TPT, k4 = threadIdx.x % TPT;
+  const int ntile = min(G, p.T - tau0);
+
+  griddep_launch();
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  griddep_wait();
+  if (threadIdx.x == 0) {
+    mbar_expect_tx(bar, kInBytes);   // the full box counts, clipped rows included
+    tma_load_3d(s_in, &mapM, bar, k0, tau0, 0);
+  }
+  const bool ok = __syncthreads_and(mbar_wait(bar, 0u, &abort_flag) ? 1 : 0) != 0;
+  if (!ok) {
+    if (threadIdx.x == 0) atomicExch(status, -6);
+    return;
+  }
+  if (g < ntile) {
+    const uint32_t rd = s_in + ((uint32_t)g * KC + 4u * (uint32_t)k4);
+    uint32_t wd[T2];
+#pragma unroll
+    for (int xi = 0; xi < T2; ++xi) wd[xi] = lds32(rd + (uint32_t)xi * (G * KC)) ^ 0x80808080u;
+    uint32_t outw[M * M];
+#pragma unroll
+    for (int i = 0; i < M * M; ++i) outw[i] = 0u;
+#pragma unroll 1
+    for (int ch = 0; ch < 4; ++ch) {
+      const int k = k0 + k4 * 4 + ch;
+      const uint32_t sel_in = 0x7440u | (uint32_t)ch;
+      const uint32_t sel_out = insert_selector(ch);
+      float Y[M * M];
+      output_transform_2d<M, MODE>(p, [&](int i, float (&mrow)[T_]) {
+#pragma unroll
+        for (int j = 0; j < T_; ++j) mrow[j] = byte_to_float_sel(wd[i * T_ + j], sel_in, 8388736.0f);
+      }, Y);
+      float b_scaled = 0.0f;
+      if (bias != nullptr) b_scaled = (float)((double)__ldg(bias + k) / (double)s_Y);
+#pragma unroll
+      for (int q = 0; q < M * M; ++q) {
+        const float yf = __fmaf_rn(Y[q], p.mult_Y, b_scaled);
+        const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
+        outw[q] = __byte_perm(outw[q], (uint32_t)(magic_to_int(r) + p.z_Y), sel_out);
+      }
+    }
+    const uint32_t wr = s_out + (uint32_t)g * kTileOut + 4u * (uint32_t)k4;
+#pragma unroll
+    for (int q = 0; q < M * M; ++q) sts32(wr + (uint32_t)q * KC, outw[q]);
+  }
+  fence_async_smem();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < ntile; ++i) {
+      const int tau = tau0 + i;
+      const int tw = tau % p.TW;
+      const int th = (tau / p.TW) % p.TH;
+      const int n = tau / (p.TW * p.TH);
+      tma_store_4d(&mapY, s_out + (uint32_t)i * kTileOut, k0, tw * M, th * M, n);
+    }
+    bulk_commit();
+    bulk_wait_all();
+  }
+}
+
+// ---------------------------------------------------------------------------
+// Launchers.  CC (or KC) is the largest of 256 / 128 / 64 that divides the
+// channel count; G makes the block at least 64 threads.
+// ---------------------------------------------------------------------------
+namespace {
+
+template <int M, int MODE, int CC, int G>
+int input_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
+                     int* status, cudaStream_t st) {
+  constexpr size_t smem = 2 * (size_t)G * (M + 2) * (M + 2) * CC + 128 + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k_input_transform_tma<M, MODE, CC, G>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return -5;
+    attr_set = true;
+  }
+  const int units = ((p.T + G - 1) / G) * (p.C / CC);
+  return launch_kernel(k_input_transform_tma<M, MODE, CC, G>, dim3((unsigned)units),
+                       dim3((CC / 4) * G), smem, st, pdl, p, mapX, mapV, status);
+}
+template <int M, int MODE>
+int input_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
+                   int* status, cudaStream_t st) {
+  const int cc = tma_chunk(p.C);
+  return cc == 256 ? input_tma_launch<M, MODE, 256, 1>(p, pdl, mapX, mapV, status, st)
+       : cc == 128 ? input_tma_launch<M, MODE, 128, 2>(p, pdl, mapX, mapV, status, st)
+                   : input_tma_launch<M, MODE, 64, 4>(p, pdl, mapX, mapV, status, st);
+}
+
+template <int M, int MODE, int KC, int G>
+int output_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapM, const CUtensorMap& mapY,
+                      const float* bias, float s_Y, int* status, cudaStream_t st) {
+  constexpr size_t smem = (size_t)G * ((M + 2) * (M + 2) + M * M) * KC + 128 + 16;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(k_output_transform_tma<M, MODE, KC, G>,
+                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+      return -5;
+    attr_set = true;
+  }
+  const int units = ((p.T + G - 1) / G) * (p.K / KC);
+  return launch_kernel(k_output_transform_tma<M, MODE, KC, G>, dim3((unsigned)units),
+                       dim3((KC / 4) * G), smem, st, pdl, p, mapM, mapY, bias, s_Y, status);
+}
+template <int M, int MODE>
+int output_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapM, const CUtensorMap& mapY,
+                    const float* bias, float s_Y, int* status, cudaStream_t st) {
+  const int kc = tma_chunk(p.K);
+  return kc == 256 ? output_tma_launch<M, MODE, 256, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+       : kc == 128 ? output_tma_launch<M, MODE, 128, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                   : output_tma_launch<M, MODE, 64, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+}
+
+}  // namespace
+
+int WINO_CAT(launch_input_transform_tma_m, WINO_M)(const Params& p, const LaunchOpt& o,
+                                                    const CUtensorMap& mapX,
+                                                    const CUtensorMap& mapV, int* status,
+                                                    cudaStream_t st) {
+  if (!o.std_mats) return input_tma_mode<WINO_M, kDense>(p, o.pdl, mapX, mapV, status, st);
+  if (WINO_M == 4) return input_tma_mode<WINO_M, kExact>(p, o.pdl, mapX, mapV, status, st);
+  return input_tma_mode<WINO_M, kSparse>(p, o.pdl, mapX, mapV, status, st);
+}
+int WINO_CAT(launch_output_transform_tma_m, WINO_M)(const Params& p, const LaunchOpt& o,
+                                                     const CUtensorMap& mapM,
+                                                     const CUtensorMap& mapY, const float* bias,
+                                                     float s_Y, int* status, cudaStream_t st) {
+  if (!o.std_mats) return output_tma_mode<WINO_M, kDense>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
+  if (WINO_M == 4) return output_tma_mode<WINO_M, kExact>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
+  return output_tma_mode<WINO_M, kSparse>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
+}
+
+}  // namespace wino

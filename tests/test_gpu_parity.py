@@ -11,7 +11,7 @@ from helpers import build_layer, small
 
 pytestmark = pytest.mark.gpu
 
-TC, DP4A, SMALLC = 1, 2, 3
+TC, DP4A, SMALLC, TC_PTR = 1, 2, 3, 4
 
 
 def _compare(L, x_q, w_q, bias, path, dumps=True):
@@ -41,12 +41,15 @@ SHAPES = [
     (3, 64, 13, 5, 64),
     (1, 160, 6, 6, 80),      # C spans two 128-byte stages with a partial one
     (5, 48, 10, 11, 272),    # K > 256: two column blocks
+    (2, 128, 9, 10, 192),    # TMA-staged transforms: 128- and 64-channel chunks, ragged tiles
+    (1, 512, 4, 4, 512),     # 256-channel chunks, two per tile
+    (3, 256, 7, 7, 128),     # odd tile count: last block of a 2-tile group is partial
 ]
 
 
 @pytest.mark.parametrize("m", [2, 4, 6])
 @pytest.mark.parametrize("shape", SHAPES)
-@pytest.mark.parametrize("path", [TC, DP4A])
+@pytest.mark.parametrize("path", [TC, TC_PTR, DP4A])
 def test_staged_paths_every_stage(m, shape, path):
     N, C, H, W, K = shape
     wl = wi.Workload("s", 3000 + m, N, C, H, W, K, m)
@@ -57,16 +60,18 @@ def test_staged_paths_every_stage(m, shape, path):
 @pytest.mark.parametrize("m", [2, 4, 6])
 @pytest.mark.parametrize("path", [TC, DP4A, SMALLC])
 def test_flex_matrices(m, path):
-    wl = wi.Workload("f", 3100 + m, 2, 32, 9, 7, 32, m, flex=True)
+    C = 32 if path == SMALLC else 64
+    wl = wi.Workload("f", 3100 + m, 2, C, 9, 7, C, m, flex=True)
     L, x_q, w_q, bias = build_layer(wl)
     _compare(L, x_q, w_q, bias, path, dumps=path != SMALLC)
 
 
 @pytest.mark.parametrize("m", [2, 4, 6])
-@pytest.mark.parametrize("path", [TC, DP4A, SMALLC])
+@pytest.mark.parametrize("path", [TC, TC_PTR, DP4A, SMALLC])
 @pytest.mark.parametrize("variant", ["no_qm", "float_out", "no_qm_float", "relu", "no_bias", "zero_points"])
 def test_variants(m, path, variant):
-    wl = wi.Workload("v", 3200 + m, 2, 16, 8, 10, 32, m)
+    C, K = (16, 32) if path == SMALLC else (64, 64)
+    wl = wi.Workload("v", 3200 + m, 2, C, 8, 10, K, m)
     kw = {}
     if variant in ("no_qm", "no_qm_float"):
         kw["q_M"] = False
@@ -117,6 +122,7 @@ def test_full_size_configs(name):
     L, x_q, w_q, bias = build_layer(wl)
     g = _compare(L, x_q, w_q, bias, TC)
     assert g["launches"] >= 4
+    _compare(L, x_q, w_q, bias, TC_PTR)
 
 
 def test_cfg3_without_qm():
