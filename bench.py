@@ -261,40 +261,53 @@ def run_ours(args, wl):
     value = units / (ms * 1e-3) / 1e12
     ms_per_step = ms / args.steps
 
-    # ---- per-kernel times for the roofline: events between the three kernels,
-    #      launches queued behind a short device-side delay so that host launch
-    #      latency is not measured ----
+    # ---- per-kernel times for the roofline: each staged kernel alone, launched
+    #      back to back from a CUDA graph on rotating buffers, CUDA events around
+    #      the replays (steady-state launch duration, host launch cost excluded) ----
     peaks = load_peaks()
     roofline = None
     stages = None
     if plan.path != binding.PATH_SMALLC:
-        nprof = 60
-        evs = []
-        for i in range(nprof):
-            four = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
-            for e in four:
-                e.record()
-            evs.append(four)
+        names = ["input_transform", "hadamard_gemm", "output_transform"]
+        us = []
+        for mask in (1, 2, 4):
+            def stage_step(i, mask=mask):
+                j = i % R
+                plan.debug_run_stages(mask, xs[j], Us[j], b_dev, ys[j], ws)
+            for i in range(3):
+                stage_step(i)
+            torch.cuda.synchronize()
+            sg = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(sg, stream=side):
+                    for i in range(2 * R):
+                        stage_step(i)
+            torch.cuda.synchronize()
+            sg.replay()
+            torch.cuda.synchronize()
+            s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            nrep = 10
+            s0.record()
+            for _ in range(nrep):
+                sg.replay()
+            s1.record()
+            torch.cuda.synchronize()
+            us.append(s0.elapsed_time(s1) * 1e3 / (nrep * 2 * R))
+        # restore the workspace contents of a complete step
+        step(0)
         torch.cuda.synchronize()
-        for i in range(nprof):
-            plan.set_stage_events([e.cuda_event for e in evs[i]])
-            torch.cuda._sleep(400000)
-            step(i)
-        plan.set_stage_events(None)
-        torch.cuda.synchronize()
-        dur = [[evs[i][k].elapsed_time(evs[i][k + 1]) * 1e3 for i in range(nprof)] for k in range(3)]
-        us = [statistics.median(d) for d in dur]
         t = wl.m + 2
         T = plan.T
         vq = t * t * T * wl.C
         mq = t * t * T * wl.K
         alg = {"input_transform": xb + vq, "hadamard_gemm": vq + plan.weight_bytes + mq,
                "output_transform": mq + yb}
-        names = ["input_transform", "hadamard_gemm", "output_transform"]
         stages = {n: {"us": u, "algorithmic_bytes": alg[n], "GBps": alg[n] / (u * 1e-6) / 1e9}
                   for n, u in zip(names, us)}
         stages["hadamard_gemm"]["wino_TOPS"] = wino_ops(wl, wl.N) / (us[1] * 1e-6) / 1e12
         dom = max(range(3), key=lambda k: us[k])
+        kernel_names = {"input_transform": "k_input_transform_tma", "hadamard_gemm": "k_gemm_tc",
+                        "output_transform": "k_output_transform_tma"}
         if dom == 1:
             peak = 2.0 * peaks["bf16_tflops"]
             ach = wino_ops(wl, wl.N) / (us[1] * 1e-6) / 1e12
@@ -304,7 +317,7 @@ def run_ours(args, wl):
         else:
             n = names[dom]
             ach = alg[n] / (us[dom] * 1e-6) / 1e9
-            roofline = {"kernel": "k_" + n, "bound": "hbm", "achieved": ach,
+            roofline = {"kernel": kernel_names[n], "bound": "hbm", "achieved": ach,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                         "traffic": None, "peak_note": f"of {peaks['source']}"}
     # whole-layer roofline of the path's definition: slower of MMA work at the int8

@@ -172,6 +172,15 @@ int wino_last_status(const wino_plan_t* plan, void* stream);
  * of that forward call. */
 int wino_debug_dump_stage(const wino_plan_t* plan, int stage, void* dst_dev, size_t bytes);
 
+/* Runs a subset of the three kernels of a staged path on the caller's buffers
+ * (stages of the paper's Fig. 2): stage_mask bit 0 = input transform (x -> V_q in
+ * the workspace), bit 1 = Hadamard GEMMs (V_q, U_q -> m_q in the workspace),
+ * bit 2 = output transform (m_q -> y).  Stages left out read whatever an earlier
+ * call left in the workspace.  For debugging and per-kernel timing. */
+int wino_debug_run_stages(const wino_plan_t* plan, int stage_mask, const int8_t* x_NHWC_dev,
+                          const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
+                          void* workspace_dev, void* stream);
+
 /* Number of kernels launched by this plan since it was created. */
 long wino_launch_count(const wino_plan_t* plan);
 

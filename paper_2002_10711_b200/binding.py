@@ -22,7 +22,7 @@ STAGE_VQ, STAGE_M_I32, STAGE_MQ = 0, 1, 2
 EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
-    "wino_conv_forward", "wino_calibrate_forward", "wino_last_status", "wino_debug_dump_stage",
+    "wino_conv_forward", "wino_calibrate_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages",
     "wino_launch_count", "wino_plan_set_stage_events", "wino_destroy", "wino_strerror",
 ]
 
@@ -65,6 +65,7 @@ def _load() -> ct.CDLL:
     lib.wino_transform_weights.argtypes = [vp, vp, vp, vp, vp]
     lib.wino_conv_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.wino_calibrate_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    lib.wino_debug_run_stages.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.wino_last_status.argtypes = [vp, vp]
     lib.wino_debug_dump_stage.argtypes = [vp, i32, vp, sz]
     lib.wino_launch_count.argtypes = [vp]
@@ -181,6 +182,12 @@ class Plan:
         _check(_lib.wino_conv_forward(self._h, _dptr(x_dev), _dptr(Uq_dev), _dptr(bias_dev),
                                       _dptr(y_dev), _dptr(workspace_dev), _stream_handle(stream)),
                "wino_conv_forward")
+
+    def debug_run_stages(self, stage_mask, x_dev, Uq_dev, bias_dev, y_dev, workspace_dev,
+                         stream=None) -> None:
+        _check(_lib.wino_debug_run_stages(self._h, stage_mask, _dptr(x_dev), _dptr(Uq_dev),
+                                          _dptr(bias_dev), _dptr(y_dev), _dptr(workspace_dev),
+                                          _stream_handle(stream)), "wino_debug_run_stages")
 
     def calibrate_forward(self, x_dev, Uq_dev, bias_dev, y_dev, workspace_dev, absmax4_dev,
                           stream=None) -> None:

@@ -73,11 +73,14 @@ int launch_gemm_dp4a(const Params& p, const LaunchOpt& o, const int8_t* Vq, cons
 //   warp 0   : TMA producer (one lane)
 //   warp 1   : tensor-memory owner; one lane issues the MMAs
 //   warps 2-17: epilogue.  Warp w reads TMEM lanes 32*(w%4) .. +31 (its hardware
-//              quadrant) and every fourth 32-column chunk, by (w-2)/4, two chunks
-//              in flight at a time.
+//              quadrant) and every fourth 32-column chunk, by (w-2)/4.
 // A stage holds 128 channels: A tile 128 x 128 B, B tile BN x 128 B; one MMA
 // consumes 32 channels.
 // ---------------------------------------------------------------------------
+
+constexpr int kEpiWarps = 16;
+constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
+
 struct GemmTcArgs {
   int BN;          // multiple of 16, <= 256
   int stages;
@@ -87,29 +90,27 @@ struct GemmTcArgs {
   int n_mblk, n_nblk, n_items;
 };
 
-constexpr int kEpiWarps = 16;
-constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
-
 template <bool SMALL>
 __device__ __forceinline__ float acc_to_float(uint32_t v) {
   if constexpr (SMALL) return small_int_to_float((int)v);
   else return __int2float_rn((int)v);
 }
 
-template <bool SMALL>
+// Epilogue of one 32-column chunk of one accumulator row.  FULL: all 32 columns
+// are inside K (no per-element guards).  STATS: track max |M| for calibration.
+template <bool SMALL, bool FULL, bool STATS>
 __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (&r)[32], int k0,
-                                               long o, int out_mode, void* out, bool want_max,
-                                               float& vmax) {
-  if (want_max) {
+                                               long o, int out_mode, void* out, float& vmax) {
+  if constexpr (STATS) {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
-      if (k0 + j < p.K) vmax = fmaxf(vmax, fabsf(__int2float_rn((int)r[j])));
+      if (FULL || k0 + j < p.K) vmax = fmaxf(vmax, fabsf(__int2float_rn((int)r[j])));
   }
   if (out_mode == kOutI32) {
     int4* dst = reinterpret_cast<int4*>(reinterpret_cast<int*>(out) + o);
 #pragma unroll
     for (int q = 0; q < 8; ++q)
-      if (k0 + q * 4 < p.K)
+      if (FULL || k0 + q * 4 < p.K)
         dst[q] = make_int4((int)r[4 * q], (int)r[4 * q + 1], (int)r[4 * q + 2], (int)r[4 * q + 3]);
   } else {
     uint32_t w[8];
@@ -124,9 +125,51 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
       w[q] = __byte_perm(lo, hi, 0x5410u);
     }
     uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(out) + o);
-    if (k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-    if (k0 + 16 < p.K) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    if (FULL || k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+    if (FULL || k0 + 16 < p.K) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
   }
+}
+
+// The epilogue warps' loop over their work items.
+template <bool SMALL, bool FULL, bool STATS>
+__device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs& a, void* out,
+                                              unsigned* absmaxM, uint32_t tmem_base,
+                                              uint32_t bar_acc_full, uint32_t bar_acc_empty,
+                                              volatile uint32_t* abort_p, int warp, int lane) {
+  const int quad = warp & 3;
+  const int sub = (warp - 2) >> 2;
+  const int per_xi = a.n_mblk * a.n_nblk;
+  float vmax = 0.0f;
+  int li = 0;
+  for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
+    const int xi = it / per_xi, rem = it - xi * per_xi;
+    const int nb = rem / a.n_mblk, mb = rem - nb * a.n_mblk;
+    const int buf = li & 1;
+    const uint32_t aph = (uint32_t)(li >> 1) & 1u;
+    if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8u * buf, aph, abort_p))) {
+      *abort_p = 1u;
+      break;
+    }
+    tc_fence_after();
+    const int tau = mb * kBM + quad * 32 + lane;
+    const bool row_ok = tau < p.T;
+    const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride) + ((uint32_t)(quad * 32) << 16);
+    // one chunk at a time per warp; the four warps of a scheduler hide each
+    // other's tensor-memory load latency
+    for (int col = sub * 32; col < a.BN; col += 128) {
+      uint32_t r0[32];
+      tmem_ld32(tacc + (uint32_t)col, r0);
+      tmem_ld_wait();
+      if (!row_ok) continue;
+      const int k0 = nb * a.BN + col;
+      const long o = ((long)xi * p.T + tau) * p.K + k0;
+      epilogue_chunk<SMALL, FULL, STATS>(p, r0, k0, o, a.out_mode, out, vmax);
+    }
+    tc_fence_before();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_acc_empty + 8u * buf);
+  }
+  if constexpr (STATS) atomic_absmax(absmaxM, vmax);
 }
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
@@ -220,49 +263,22 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
       }
     }
   } else {
-    // epilogue warps
-    const int quad = warp & 3;
-    const int sub = (warp - 2) >> 2;
-    const bool small = p.C <= 260;   // |M| <= 127^2 * C < 2^22
-    const bool want_max = absmaxM != nullptr;
-    float vmax = 0.0f;
-    int li = 0;
-    for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
-      const int xi = it / per_xi, rem = it - xi * per_xi;
-      const int nb = rem / a.n_mblk, mb = rem - nb * a.n_mblk;
-      const int buf = li & 1;
-      const uint32_t aph = (uint32_t)(li >> 1) & 1u;
-      if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8u * buf, aph, abort_p))) {
-        *abort_p = 1u;
-        break;
-      }
-      tc_fence_after();
-      const int tau = mb * kBM + quad * 32 + lane;
-      const bool row_ok = tau < p.T;
-      const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride) + ((uint32_t)(quad * 32) << 16);
-      for (int col = sub * 32; col < a.BN; col += 256) {
-        // two chunks in flight: col and col + 128
-        const bool two = col + 128 < a.BN;
-        uint32_t r0[32], r1[32];
-        tmem_ld32(tacc + (uint32_t)col, r0);
-        if (two) tmem_ld32(tacc + (uint32_t)(col + 128), r1);
-        tmem_ld_wait();
-        if (!row_ok) continue;
-        const int k0 = nb * a.BN + col;
-        const long o = ((long)xi * p.T + tau) * p.K + k0;
-        if (small) {
-          epilogue_chunk<true>(p, r0, k0, o, a.out_mode, out, want_max, vmax);
-          if (two) epilogue_chunk<true>(p, r1, k0 + 128, o + 128, a.out_mode, out, want_max, vmax);
-        } else {
-          epilogue_chunk<false>(p, r0, k0, o, a.out_mode, out, want_max, vmax);
-          if (two) epilogue_chunk<false>(p, r1, k0 + 128, o + 128, a.out_mode, out, want_max, vmax);
-        }
-      }
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(bar_acc_empty + 8u * buf);
-    }
-    if (want_max) atomic_absmax(absmaxM, vmax);
+    // epilogue warps.  small: |M| <= 127^2 * C < 2^22; full: every 32-column chunk
+    // lies inside K.
+    const bool small = p.C <= 260;
+    const bool full = (p.K % 32) == 0 && (a.BN % 32) == 0;
+    if (absmaxM != nullptr)
+      epilogue_loop<false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
+                                        abort_p, warp, lane);
+    else if (small && full)
+      epilogue_loop<true, true, false>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
+                                       abort_p, warp, lane);
+    else if (full)
+      epilogue_loop<false, true, false>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
+                                        abort_p, warp, lane);
+    else
+      epilogue_loop<false, false, false>(p, a, out, absmaxM, tmem_base, bar_acc_full,
+                                         bar_acc_empty, abort_p, warp, lane);
   }
   __syncwarp();
   tc_fence_before();

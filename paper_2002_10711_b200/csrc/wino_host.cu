@@ -209,8 +209,9 @@ int launch_gemm(const wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void*
                         pl->status_dev, st);
 }
 
+// stage_mask: bit 0 input transform, bit 1 Hadamard GEMMs, bit 2 output transform
 int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias, void* y,
-                 void* ws, unsigned* absmax4, cudaStream_t st) {
+                 void* ws, unsigned* absmax4, cudaStream_t st, int stage_mask = 7) {
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
   const bool calib = absmax4 != nullptr;
   const bool pdl = pl->pdl && !calib;
@@ -232,10 +233,10 @@ int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const
   }
   const bool ev = pl->stage_ev_on;
   if (ev) cudaEventRecord(pl->stage_ev[0], st);
-  pl->launches++;
   const bool tma_ok = pl->path == WINO_PATH_STAGED_TC && !calib;
-  int rc;
-  if (tma_ok && pl->p.z_x == 0 && tma_chunk(pl->p.C) != 0) {
+  int rc = WINO_OK;
+  if (!(stage_mask & 1)) {
+  } else if (pl->launches++, tma_ok && pl->p.z_x == 0 && tma_chunk(pl->p.C) != 0) {
     const CUtensorMap* mx = map_x(pl, x);
     const CUtensorMap* mv = map_stage(pl, pl->cache_vst, Vq, pl->p.C);
     if (mx == nullptr || mv == nullptr) return WINO_ERR_CUDA;
@@ -246,15 +247,17 @@ int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const
   }
   if (rc != WINO_OK) return rc;
   if (ev) cudaEventRecord(pl->stage_ev[1], st);
-  rc = launch_gemm(run, Vq, Uq, mbuf, pl->p.qM_enabled ? kOutMq : kOutI32,
-                   calib ? absmax4 + 1 : nullptr, pdl && !ev, st);
-  if (run != pl) {
-    pl->launches++;
+  if (stage_mask & 2) {
+    rc = launch_gemm(run, Vq, Uq, mbuf, pl->p.qM_enabled ? kOutMq : kOutI32,
+                     calib ? absmax4 + 1 : nullptr, pdl && !ev, st);
+    if (run != pl) {
+      pl->launches++;
+    }
   }
   if (rc != WINO_OK) return rc;
   if (ev) cudaEventRecord(pl->stage_ev[2], st);
-  pl->launches++;
-  if (tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
+  if (!(stage_mask & 4)) {
+  } else if (pl->launches++, tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
     const CUtensorMap* mm = map_stage(pl, pl->cache_mld, mbuf, pl->p.K);
     const CUtensorMap* my = map_y(pl, y);
     if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
@@ -406,6 +409,16 @@ int wino_calibrate_forward(const wino_plan_t* pl, const int8_t* x, const int8_t*
   if (!aligned16(x) || !aligned16(Uq) || (y && !aligned16(y)) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
   return forward_impl(pl, x, Uq, bias, y, ws, absmax4, (cudaStream_t)stream);
+}
+
+int wino_debug_run_stages(const wino_plan_t* pl, int stage_mask, const int8_t* x, const int8_t* Uq,
+                          const float* bias, void* y, void* ws, void* stream) {
+  if (pl == nullptr || x == nullptr || Uq == nullptr || y == nullptr) return WINO_ERR_INVALID;
+  if (stage_mask < 1 || stage_mask > 7) return WINO_ERR_INVALID;
+  if (pl->path == WINO_PATH_SMALLC) return WINO_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(Uq) || !aligned16(y) || (bias && !aligned16(bias)))
+    return WINO_ERR_ALIGNMENT;
+  return forward_impl(pl, x, Uq, bias, y, ws, nullptr, (cudaStream_t)stream, stage_mask);
 }
 
 int wino_last_status(const wino_plan_t* pl, void* stream) {

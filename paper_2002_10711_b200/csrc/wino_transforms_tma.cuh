@@ -15,11 +15,28 @@
 
 namespace wino {
 
-template <int M, int MODE, int CC, int G>
-__global__ void __launch_bounds__((CC / 4) * G)
+template <int CPT>
+__device__ __forceinline__ uint32_t lds_pack(uint32_t addr) {
+  if constexpr (CPT == 4) return lds32(addr);
+  else {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
+    return (uint32_t)v;
+  }
+}
+template <int CPT>
+__device__ __forceinline__ void sts_pack(uint32_t addr, uint32_t v) {
+  if constexpr (CPT == 4) sts32(addr, v);
+  else {
+    asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+  }
+}
+
+template <int M, int MODE, int CC, int G, int CPT>
+__global__ void __launch_bounds__((CC / CPT) * G)
 k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
                       const __grid_constant__ CUtensorMap mapV, int* __restrict__ status) {
-  constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / 4;
+  constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
   constexpr uint32_t kUnitBytes = G * kTileBytes;
   extern __shared__ uint8_t smem_raw[];
@@ -60,15 +77,15 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
     return;
   }
   if (g < ntile) {
-    const uint32_t rd = s_in + (uint32_t)g * kTileBytes + 4u * (uint32_t)c4;
+    const uint32_t rd = s_in + (uint32_t)g * kTileBytes + (uint32_t)(CPT * c4);
     uint32_t wd[T2];
 #pragma unroll
-    for (int ab = 0; ab < T2; ++ab) wd[ab] = lds32(rd + (uint32_t)ab * CC) ^ 0x80808080u;
+    for (int ab = 0; ab < T2; ++ab) wd[ab] = lds_pack<CPT>(rd + (uint32_t)ab * CC) ^ 0x80808080u;
     uint32_t out[T2];
 #pragma unroll
     for (int i = 0; i < T2; ++i) out[i] = 0u;
 #pragma unroll 1
-    for (int ch = 0; ch < 4; ++ch) {
+    for (int ch = 0; ch < CPT; ++ch) {
       const uint32_t sel_in = 0x7440u | (uint32_t)ch;
       const uint32_t sel_out = insert_selector(ch);
       float V[T2];
@@ -82,9 +99,9 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
         out[xi] = __byte_perm(out[xi], __float_as_uint(r), sel_out);
       }
     }
-    const uint32_t wr = s_out + ((uint32_t)g * CC + 4u * (uint32_t)c4);
+    const uint32_t wr = s_out + ((uint32_t)g * CC + (uint32_t)(CPT * c4));
 #pragma unroll
-    for (int xi = 0; xi < T2; ++xi) sts32(wr + (uint32_t)xi * (G * CC), out[xi]);
+    for (int xi = 0; xi < T2; ++xi) sts_pack<CPT>(wr + (uint32_t)xi * (G * CC), out[xi]);
   }
   fence_async_smem();
   __syncthreads();
@@ -95,12 +112,12 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   }
 }
 
-template <int M, int MODE, int KC, int G>
-__global__ void __launch_bounds__((KC / 4) * G)
+template <int M, int MODE, int KC, int G, int CPT>
+__global__ void __launch_bounds__((KC / CPT) * G)
 k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapM,
                        const __grid_constant__ CUtensorMap mapY, const float* __restrict__ bias,
                        float s_Y, int* __restrict__ status) {
-  constexpr int T_ = M + 2, T2 = T_ * T_, TPT = KC / 4;
+  constexpr int T_ = M + 2, T2 = T_ * T_, TPT = KC / CPT;
   constexpr uint32_t kInBytes = T2 * G * KC;          // [T2][G][KC]
   constexpr uint32_t kTileOut = M * M * KC;           // [M][M][KC] per tile
   extern __shared__ uint8_t smem_raw[];
@@ -135,16 +152,16 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     return;
   }
   if (g < ntile) {
-    const uint32_t rd = s_in + ((uint32_t)g * KC + 4u * (uint32_t)k4);
+    const uint32_t rd = s_in + ((uint32_t)g * KC + (uint32_t)(CPT * k4));
     uint32_t wd[T2];
 #pragma unroll
-    for (int xi = 0; xi < T2; ++xi) wd[xi] = lds32(rd + (uint32_t)xi * (G * KC)) ^ 0x80808080u;
+    for (int xi = 0; xi < T2; ++xi) wd[xi] = lds_pack<CPT>(rd + (uint32_t)xi * (G * KC)) ^ 0x80808080u;
     uint32_t outw[M * M];
 #pragma unroll
     for (int i = 0; i < M * M; ++i) outw[i] = 0u;
 #pragma unroll 1
-    for (int ch = 0; ch < 4; ++ch) {
-      const int k = k0 + k4 * 4 + ch;
+    for (int ch = 0; ch < CPT; ++ch) {
+      const int k = k0 + k4 * CPT + ch;
       const uint32_t sel_in = 0x7440u | (uint32_t)ch;
       const uint32_t sel_out = insert_selector(ch);
       float Y[M * M];
@@ -161,9 +178,9 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
         outw[q] = __byte_perm(outw[q], (uint32_t)(magic_to_int(r) + p.z_Y), sel_out);
       }
     }
-    const uint32_t wr = s_out + (uint32_t)g * kTileOut + 4u * (uint32_t)k4;
+    const uint32_t wr = s_out + (uint32_t)g * kTileOut + (uint32_t)(CPT * k4);
 #pragma unroll
-    for (int q = 0; q < M * M; ++q) sts32(wr + (uint32_t)q * KC, outw[q]);
+    for (int q = 0; q < M * M; ++q) sts_pack<CPT>(wr + (uint32_t)q * KC, outw[q]);
   }
   fence_async_smem();
   __syncthreads();
@@ -186,52 +203,68 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
 // ---------------------------------------------------------------------------
 namespace {
 
-template <int M, int MODE, int CC, int G>
+// Channels per thread: 4 when that already gives every SM a dozen warps, else 2
+// (shorter serial chains per thread for small problems).
+inline int tma_cpt(long tiles_times_channels) {
+  static const int forced = [] { const char* e = getenv("WINO_TMA_CPT"); return e ? atoi(e) : 0; }();
+  if (forced == 2 || forced == 4) return forced;
+  return tiles_times_channels / (4 * 32) >= 148l * 16 ? 4 : 2;
+}
+
+template <int M, int MODE, int CC, int G, int CPT>
 int input_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
                      int* status, cudaStream_t st) {
   constexpr size_t smem = 2 * (size_t)G * (M + 2) * (M + 2) * CC + 128 + 16;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(k_input_transform_tma<M, MODE, CC, G>,
+    if (cudaFuncSetAttribute(k_input_transform_tma<M, MODE, CC, G, CPT>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return -5;
     attr_set = true;
   }
   const int units = ((p.T + G - 1) / G) * (p.C / CC);
-  return launch_kernel(k_input_transform_tma<M, MODE, CC, G>, dim3((unsigned)units),
-                       dim3((CC / 4) * G), smem, st, pdl, p, mapX, mapV, status);
+  return launch_kernel(k_input_transform_tma<M, MODE, CC, G, CPT>, dim3((unsigned)units),
+                       dim3((CC / CPT) * G), smem, st, pdl, p, mapX, mapV, status);
 }
 template <int M, int MODE>
 int input_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
                    int* status, cudaStream_t st) {
   const int cc = tma_chunk(p.C);
-  return cc == 256 ? input_tma_launch<M, MODE, 256, 1>(p, pdl, mapX, mapV, status, st)
-       : cc == 128 ? input_tma_launch<M, MODE, 128, 2>(p, pdl, mapX, mapV, status, st)
-                   : input_tma_launch<M, MODE, 64, 4>(p, pdl, mapX, mapV, status, st);
+  if (tma_cpt((long)p.T * p.C) == 4)
+    return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 4>(p, pdl, mapX, mapV, status, st)
+         : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 4>(p, pdl, mapX, mapV, status, st)
+                     : input_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapX, mapV, status, st);
+  return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 2>(p, pdl, mapX, mapV, status, st)
+       : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 2>(p, pdl, mapX, mapV, status, st)
+                   : input_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapX, mapV, status, st);
 }
 
-template <int M, int MODE, int KC, int G>
+template <int M, int MODE, int KC, int G, int CPT>
 int output_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapM, const CUtensorMap& mapY,
                       const float* bias, float s_Y, int* status, cudaStream_t st) {
   constexpr size_t smem = (size_t)G * ((M + 2) * (M + 2) + M * M) * KC + 128 + 16;
   static bool attr_set = false;
   if (!attr_set) {
-    if (cudaFuncSetAttribute(k_output_transform_tma<M, MODE, KC, G>,
+    if (cudaFuncSetAttribute(k_output_transform_tma<M, MODE, KC, G, CPT>,
                              cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
       return -5;
     attr_set = true;
   }
   const int units = ((p.T + G - 1) / G) * (p.K / KC);
-  return launch_kernel(k_output_transform_tma<M, MODE, KC, G>, dim3((unsigned)units),
-                       dim3((KC / 4) * G), smem, st, pdl, p, mapM, mapY, bias, s_Y, status);
+  return launch_kernel(k_output_transform_tma<M, MODE, KC, G, CPT>, dim3((unsigned)units),
+                       dim3((KC / CPT) * G), smem, st, pdl, p, mapM, mapY, bias, s_Y, status);
 }
 template <int M, int MODE>
 int output_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapM, const CUtensorMap& mapY,
                     const float* bias, float s_Y, int* status, cudaStream_t st) {
   const int kc = tma_chunk(p.K);
-  return kc == 256 ? output_tma_launch<M, MODE, 256, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-       : kc == 128 ? output_tma_launch<M, MODE, 128, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                   : output_tma_launch<M, MODE, 64, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+  if (tma_cpt((long)p.T * p.K) == 4)
+    return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+         : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                     : output_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+  return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+       : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                   : output_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st);
 }
 
 }  // namespace
