@@ -151,6 +151,37 @@ int wino_conv_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev, const i
                       const float* bias_K_dev, void* y_NHWK_dev, void* workspace_dev,
                       void* stream);
 
+/* Largest workspace wino_conv_forward_static can serve, in bytes. */
+#define WINO_STATIC_SCRATCH_BYTES (20u * 1024u * 1024u)
+
+/* wino_conv_forward for callers that cannot hand over a workspace because they
+ * cannot allocate device memory at this point.  (The paper has no counterpart:
+ * this is a deployment convenience of this library.)  Typical cases: a plug-in
+ * inside a host framework that owns all device memory through its own pool and
+ * does not let plug-ins call the CUDA allocator; a latency-critical serving
+ * loop, where cudaMalloc may block on the whole device and can fail late under
+ * a fixed memory budget; start-up code that runs before the application's
+ * allocator exists.
+ *
+ * Same arguments, results and errors as wino_conv_forward, minus the workspace:
+ * V_q and m_q live in a static device array of WINO_STATIC_SCRATCH_BYTES built
+ * into the library (every GPU that loads the library holds those bytes until
+ * the process exits).  A plan whose wino_workspace_bytes exceeds that size is
+ * refused with WINO_ERR_WORKSPACE and nothing is launched.  The call makes no
+ * cudaMalloc / cudaFree and uses no allocating library routine.
+ *
+ * First use on a device: the first call made with a given device current looks
+ * up the array's device address (cudaGetSymbolAddress) and remembers it; make
+ * that first call before starting any stream capture on that device.
+ * Sharing: all calls on a device, from every plan and stream, use the same
+ * array, and it keeps whatever the last call left there.  Nothing in it has to
+ * start at zero (each call overwrites every byte it later reads).  Two calls
+ * whose kernels overlap on the GPU (different streams, no ordering between
+ * them) race on the array and corrupt each other's result: order them. */
+int wino_conv_forward_static(const wino_plan_t* plan, const int8_t* x_NHWC_dev,
+                             const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
+                             void* stream);
+
 /* Calibration pass (paper: Table 1 caption, range "warmup"; here a one-shot
  * max-abs): runs the forward pass on a staged path and records, as float bits
  * in absmax4_dev[0..3] (device, caller-zeroed uint32[4]), the max-abs of

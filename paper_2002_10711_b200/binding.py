@@ -18,11 +18,12 @@ WINO_OK = 0
 ERR_INVALID, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
 PATH_AUTO, PATH_STAGED_TC, PATH_STAGED_DP4A, PATH_SMALLC, PATH_STAGED_TC_PTR = 0, 1, 2, 3, 4
 STAGE_VQ, STAGE_M_I32, STAGE_MQ = 0, 1, 2
+STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
 
 EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
-    "wino_conv_forward", "wino_calibrate_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages",
+    "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages",
     "wino_launch_count", "wino_plan_set_stage_events", "wino_destroy", "wino_strerror",
 ]
 
@@ -64,6 +65,7 @@ def _load() -> ct.CDLL:
     lib.wino_plan_multipliers.argtypes = [vp, vp]
     lib.wino_transform_weights.argtypes = [vp, vp, vp, vp, vp]
     lib.wino_conv_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.wino_conv_forward_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.wino_calibrate_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.wino_debug_run_stages.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.wino_last_status.argtypes = [vp, vp]
@@ -182,6 +184,13 @@ class Plan:
         _check(_lib.wino_conv_forward(self._h, _dptr(x_dev), _dptr(Uq_dev), _dptr(bias_dev),
                                       _dptr(y_dev), _dptr(workspace_dev), _stream_handle(stream)),
                "wino_conv_forward")
+
+    def conv_forward_static(self, x_dev, Uq_dev, bias_dev, y_dev, stream=None) -> None:
+        """wino_conv_forward_static: no workspace argument; the library's built-in static
+        scratch (STATIC_SCRATCH_BYTES at most) is used, and nothing is allocated."""
+        _check(_lib.wino_conv_forward_static(self._h, _dptr(x_dev), _dptr(Uq_dev), _dptr(bias_dev),
+                                             _dptr(y_dev), _stream_handle(stream)),
+               "wino_conv_forward_static")
 
     def debug_run_stages(self, stage_mask, x_dev, Uq_dev, bias_dev, y_dev, workspace_dev,
                          stream=None) -> None:

@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include <cuda.h>
@@ -62,7 +63,36 @@ struct wino_plan {
   bool stage_ev_on;
 };
 
+// Scratch of wino_conv_forward_static: V_q and m_q of one layer call.  A plain
+// file-scope device array, so every GPU that loads this library holds these
+// bytes from module load until the process exits.  In host code the name below
+// is only a handle; the device address is looked up once per device with
+// cudaGetSymbolAddress and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[WINO_STATIC_SCRATCH_BYTES];
+
 namespace {
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {nullptr};
+std::mutex g_static_scratch_mutex;
+
+// Device address of the static scratch on the current device (looked up on the
+// first call for that device, with that device current).
+int static_scratch_address(void** out) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return WINO_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* ptr = nullptr;
+    if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || ptr == nullptr) {
+      cudaGetLastError();
+      return WINO_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = ptr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return WINO_OK;
+}
 
 EncodeTiledFn get_encode_fn() {
   static EncodeTiledFn fn = nullptr;
@@ -401,6 +431,18 @@ int wino_conv_forward(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, 
   if (!aligned16(x) || !aligned16(Uq) || !aligned16(y) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
   return forward_impl(pl, x, Uq, bias, y, ws, nullptr, (cudaStream_t)stream);
+}
+
+int wino_conv_forward_static(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq,
+                             const float* bias, void* y, void* stream) {
+  if (pl == nullptr || x == nullptr || Uq == nullptr || y == nullptr) return WINO_ERR_INVALID;
+  if (!aligned16(x) || !aligned16(Uq) || !aligned16(y) || (bias && !aligned16(bias)))
+    return WINO_ERR_ALIGNMENT;
+  if (wino_workspace_bytes(pl) > (size_t)WINO_STATIC_SCRATCH_BYTES) return WINO_ERR_WORKSPACE;
+  void* scratch = nullptr;
+  const int rc = static_scratch_address(&scratch);
+  if (rc != WINO_OK) return rc;
+  return forward_impl(pl, x, Uq, bias, y, scratch, nullptr, (cudaStream_t)stream);
 }
 
 int wino_calibrate_forward(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq,
