@@ -33,6 +33,12 @@ if ROOT not in sys.path:
 
 import wino_inputs as wi  # noqa: E402
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
+# summarised in profiles/cfg3_staged_tc_launches_and_kernels.md; valid for cfg3 and for the
+# kernels as profiled there (set an entry to None when its kernel changes).
+NCU_TRAFFIC_CFG3 = {"k_input_transform_tma": 4.21e6, "k_gemm_tc": 11.84e6,
+                    "k_output_transform_tma": 9.45e6}
+
 METRIC = "effective direct-conv-equivalent int8 TOPS (Winograd-aware quantized 3x3 conv forward)"
 UNIT = "TOPS"
 
@@ -312,14 +318,16 @@ def run_ours(args, wl):
             peak = 2.0 * peaks["bf16_tflops"]
             ach = wino_ops(wl, wl.N) / (us[1] * 1e-6) / 1e12
             roofline = {"kernel": "k_gemm_tc", "bound": "tensor", "achieved": ach, "peak": peak,
-                        "unit": "TOP/s", "frac": ach / peak, "traffic": None,
+                        "unit": "TOP/s", "frac": ach / peak,
+                        "traffic": NCU_TRAFFIC_CFG3.get("k_gemm_tc") if wl.name == "cfg3" else None,
                         "peak_note": f"int8 = 2 x {peaks['source']} bf16 burst peak"}
         else:
             n = names[dom]
             ach = alg[n] / (us[dom] * 1e-6) / 1e9
             roofline = {"kernel": kernel_names[n], "bound": "hbm", "achieved": ach,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                        "traffic": None, "peak_note": f"of {peaks['source']}"}
+                        "traffic": NCU_TRAFFIC_CFG3.get(kernel_names[n]) if wl.name == "cfg3" else None,
+                        "peak_note": f"of {peaks['source']}"}
     # whole-layer roofline of the path's definition: slower of MMA work at the int8
     # tensor peak and algorithmic bytes (x + y + U_q) at the HBM peak
     t_mma = wino_ops(wl, wl.N) / (2.0 * peaks["bf16_tflops"] * 1e12)
