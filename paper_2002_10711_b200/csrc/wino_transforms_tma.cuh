@@ -18,17 +18,23 @@ namespace wino {
 template <int CPT>
 __device__ __forceinline__ uint32_t lds_pack(uint32_t addr) {
   if constexpr (CPT == 4) return lds32(addr);
-  else {
+  else if constexpr (CPT == 2) {
     uint16_t v;
     asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(addr));
     return (uint32_t)v;
+  } else {
+    uint32_t v;   // one channel per thread: the sign-extended code itself
+    asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
   }
 }
 template <int CPT>
 __device__ __forceinline__ void sts_pack(uint32_t addr, uint32_t v) {
   if constexpr (CPT == 4) sts32(addr, v);
-  else {
+  else if constexpr (CPT == 2) {
     asm volatile("st.shared.u16 [%0], %1;" ::"r"(addr), "h"((uint16_t)v) : "memory");
+  } else {
+    asm volatile("st.shared.u8 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
   }
 }
 
@@ -60,8 +66,8 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  griddep_wait();
   if (threadIdx.x == 0) {
+    griddep_wait();   // only this thread reads or writes buffers that other kernels touch
     mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
     for (int i = 0; i < ntile; ++i) {
       const int tau = tau0 + i;
@@ -70,17 +76,21 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
       const int n = tau / (p.TW * p.TH);
       tma_load_4d(s_in + (uint32_t)i * kTileBytes, &mapX, bar, c0, tw * M - 1, th * M - 1, n);
     }
+    // one thread polls (bounded); the others sleep in the barrier below
+    if (!mbar_wait(bar, 0u, &abort_flag)) {
+      abort_flag = 1u;
+      atomicExch(status, -6);  // WINO_ERR_TIMEOUT
+    }
   }
-  const bool ok = __syncthreads_and(mbar_wait(bar, 0u, &abort_flag) ? 1 : 0) != 0;
-  if (!ok) {
-    if (threadIdx.x == 0) atomicExch(status, -6);  // WINO_ERR_TIMEOUT
-    return;
-  }
+  __syncthreads();
+  if (*(volatile uint32_t*)&abort_flag != 0u) return;
+  (void)mbar_try_wait(bar, 0u);   // every thread observes the completed phase itself
   if (g < ntile) {
     const uint32_t rd = s_in + (uint32_t)g * kTileBytes + (uint32_t)(CPT * c4);
     uint32_t wd[T2];
 #pragma unroll
-    for (int ab = 0; ab < T2; ++ab) wd[ab] = lds_pack<CPT>(rd + (uint32_t)ab * CC) ^ 0x80808080u;
+    for (int ab = 0; ab < T2; ++ab)
+      wd[ab] = lds_pack<CPT>(rd + (uint32_t)ab * CC) ^ (CPT == 1 ? 0u : 0x80808080u);
     uint32_t out[T2];
 #pragma unroll
     for (int i = 0; i < T2; ++i) out[i] = 0u;
@@ -91,12 +101,14 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
       float V[T2];
       input_transform_2d<M, MODE>(p, [&](int l, float (&dcol)[T_]) {
 #pragma unroll
-        for (int a = 0; a < T_; ++a) dcol[a] = byte_to_float_sel(wd[a * T_ + l], sel_in, 8388736.0f);
+        for (int a = 0; a < T_; ++a)
+          dcol[a] = CPT == 1 ? small_int_to_float((int)wd[a * T_ + l])
+                             : byte_to_float_sel(wd[a * T_ + l], sel_in, 8388736.0f);
       }, V);
 #pragma unroll
       for (int xi = 0; xi < T2; ++xi) {
         const float r = quant_magic(V[xi], p.mult_V, p.lo_V, p.hi_V);
-        out[xi] = __byte_perm(out[xi], __float_as_uint(r), sel_out);
+        out[xi] = CPT == 1 ? __float_as_uint(r) : __byte_perm(out[xi], __float_as_uint(r), sel_out);
       }
     }
     const uint32_t wr = s_out + ((uint32_t)g * CC + (uint32_t)(CPT * c4));
@@ -108,7 +120,7 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   if (threadIdx.x == 0) {
     tma_store_3d(&mapV, s_out, c0, tau0, 0);
     bulk_commit();
-    bulk_wait_all();
+    bulk_wait_read();   // shared memory may be released; the grid's completion publishes the data
   }
 }
 
@@ -141,21 +153,24 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
-  griddep_wait();
   if (threadIdx.x == 0) {
+    griddep_wait();
     mbar_expect_tx(bar, kInBytes);   // the full box counts, clipped rows included
     tma_load_3d(s_in, &mapM, bar, k0, tau0, 0);
+    if (!mbar_wait(bar, 0u, &abort_flag)) {
+      abort_flag = 1u;
+      atomicExch(status, -6);  // WINO_ERR_TIMEOUT
+    }
   }
-  const bool ok = __syncthreads_and(mbar_wait(bar, 0u, &abort_flag) ? 1 : 0) != 0;
-  if (!ok) {
-    if (threadIdx.x == 0) atomicExch(status, -6);
-    return;
-  }
+  __syncthreads();
+  if (*(volatile uint32_t*)&abort_flag != 0u) return;
+  (void)mbar_try_wait(bar, 0u);
   if (g < ntile) {
     const uint32_t rd = s_in + ((uint32_t)g * KC + (uint32_t)(CPT * k4));
     uint32_t wd[T2];
 #pragma unroll
-    for (int xi = 0; xi < T2; ++xi) wd[xi] = lds_pack<CPT>(rd + (uint32_t)xi * (G * KC)) ^ 0x80808080u;
+    for (int xi = 0; xi < T2; ++xi)
+      wd[xi] = lds_pack<CPT>(rd + (uint32_t)xi * (G * KC)) ^ (CPT == 1 ? 0u : 0x80808080u);
     uint32_t outw[M * M];
 #pragma unroll
     for (int i = 0; i < M * M; ++i) outw[i] = 0u;
@@ -167,7 +182,9 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
       float Y[M * M];
       output_transform_2d<M, MODE>(p, [&](int i, float (&mrow)[T_]) {
 #pragma unroll
-        for (int j = 0; j < T_; ++j) mrow[j] = byte_to_float_sel(wd[i * T_ + j], sel_in, 8388736.0f);
+        for (int j = 0; j < T_; ++j)
+          mrow[j] = CPT == 1 ? small_int_to_float((int)wd[i * T_ + j])
+                             : byte_to_float_sel(wd[i * T_ + j], sel_in, 8388736.0f);
       }, Y);
       float b_scaled = 0.0f;
       if (bias != nullptr) b_scaled = (float)((double)__ldg(bias + k) / (double)s_Y);
@@ -175,7 +192,8 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
       for (int q = 0; q < M * M; ++q) {
         const float yf = __fmaf_rn(Y[q], p.mult_Y, b_scaled);
         const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
-        outw[q] = __byte_perm(outw[q], (uint32_t)(magic_to_int(r) + p.z_Y), sel_out);
+        const uint32_t code = (uint32_t)(magic_to_int(r) + p.z_Y);
+        outw[q] = CPT == 1 ? code : __byte_perm(outw[q], code, sel_out);
       }
     }
     const uint32_t wr = s_out + (uint32_t)g * kTileOut + (uint32_t)(CPT * k4);
@@ -193,7 +211,7 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
       tma_store_4d(&mapY, s_out + (uint32_t)i * kTileOut, k0, tw * M, th * M, n);
     }
     bulk_commit();
-    bulk_wait_all();
+    bulk_wait_read();
   }
 }
 
@@ -203,12 +221,13 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
 // ---------------------------------------------------------------------------
 namespace {
 
-// Channels per thread: 4 when that already gives every SM a dozen warps, else 2
-// (shorter serial chains per thread for small problems).
+// Channels per thread.  One channel per thread needs the fewest registers (so the
+// most resident warps) and no byte-insert step; it is used unless the grid is so
+// large that four channels per thread still fill every SM many warps deep.
 inline int tma_cpt(long tiles_times_channels) {
   static const int forced = [] { const char* e = getenv("WINO_TMA_CPT"); return e ? atoi(e) : 0; }();
-  if (forced == 2 || forced == 4) return forced;
-  return tiles_times_channels / (4 * 32) >= 148l * 16 ? 4 : 2;
+  if (forced == 1 || forced == 2 || forced == 4) return forced;
+  return tiles_times_channels / (4 * 32) >= 148l * 64 ? 4 : 1;
 }
 
 template <int M, int MODE, int CC, int G, int CPT>
@@ -234,6 +253,10 @@ int input_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapX, const CUt
     return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 4>(p, pdl, mapX, mapV, status, st)
          : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 4>(p, pdl, mapX, mapV, status, st)
                      : input_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapX, mapV, status, st);
+  if (tma_cpt((long)p.T * p.C) == 1)
+    return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 1>(p, pdl, mapX, mapV, status, st)
+         : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 1>(p, pdl, mapX, mapV, status, st)
+                     : input_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapX, mapV, status, st);
   return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 2>(p, pdl, mapX, mapV, status, st)
        : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 2>(p, pdl, mapX, mapV, status, st)
                    : input_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapX, mapV, status, st);
@@ -262,6 +285,10 @@ int output_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapM, const CU
     return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
          : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
                      : output_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+  if (tma_cpt((long)p.T * p.K) == 1)
+    return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+         : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                     : output_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st);
   return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
        : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
                    : output_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st);
