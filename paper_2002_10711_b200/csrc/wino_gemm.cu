@@ -87,7 +87,8 @@ struct GemmTcArgs {
   int tmem_cols;   // power of two >= 32, >= 2 * acc_stride
   int acc_stride;  // columns between the two accumulator buffers
   int out_mode;
-  int n_mblk, n_nblk, n_items;
+  int MB;          // m-blocks (128 tiles each) per work item, sharing one U_q tile
+  int n_mblk, n_nblk, n_items;   // n_mblk counts groups of MB m-blocks
 };
 
 template <bool SMALL>
@@ -151,17 +152,19 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
       break;
     }
     tc_fence_after();
-    const int tau = mb * kBM + quad * 32 + lane;
-    const bool row_ok = tau < p.T;
     const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride) + ((uint32_t)(quad * 32) << 16);
-    // one chunk at a time per warp; the four warps of a scheduler hide each
-    // other's tensor-memory load latency
-    for (int col = sub * 32; col < a.BN; col += 128) {
+    // the accumulator holds MB blocks of BN columns side by side; one chunk at a
+    // time per warp, the four warps of a scheduler hide each other's
+    // tensor-memory load latency
+    for (int col = sub * 32; col < a.MB * a.BN; col += 128) {
       uint32_t r0[32];
       tmem_ld32(tacc + (uint32_t)col, r0);
       tmem_ld_wait();
-      if (!row_ok) continue;
-      const int k0 = nb * a.BN + col;
+      const int j = a.MB > 1 ? col / a.BN : 0;
+      const int kcol = col - j * a.BN;
+      const int tau = (mb * a.MB + j) * kBM + quad * 32 + lane;
+      if (tau >= p.T) continue;
+      const int k0 = nb * a.BN + kcol;
       const long o = ((long)xi * p.T + tau) * p.K + k0;
       epilogue_chunk<SMALL, FULL, STATS>(p, r0, k0, o, a.out_mode, out, vmax);
     }
@@ -180,7 +183,7 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
   // tiles need 1024-byte alignment for the 128-byte swizzle
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t a_bytes = kBM * kStageK, b_bytes = (uint32_t)a.BN * kStageK;
-  const uint32_t stage_bytes = a_bytes + b_bytes;
+  const uint32_t stage_bytes = (uint32_t)a.MB * a_bytes + b_bytes;
   const uint32_t bars = base + (uint32_t)a.stages * stage_bytes;
   const uint32_t bar_full = bars;                           // stages x 8 B
   const uint32_t bar_empty = bar_full + 8u * a.stages;      // stages x 8 B
@@ -227,8 +230,11 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
           if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
           const uint32_t sa = base + (uint32_t)s * stage_bytes;
           mbar_expect_tx(bar_full + 8u * s, stage_bytes);
-          tma_load_3d(sa, &mapV, bar_full + 8u * s, kb * kStageK, mb * kBM, xi);
-          tma_load_3d(sa + a_bytes, &mapU, bar_full + 8u * s, kb * kStageK, nb * a.BN, xi);
+          for (int j = 0; j < a.MB; ++j)   // rows past T are filled with zeros by the TMA unit
+            tma_load_3d(sa + (uint32_t)j * a_bytes, &mapV, bar_full + 8u * s, kb * kStageK,
+                        (mb * a.MB + j) * kBM, xi);
+          tma_load_3d(sa + (uint32_t)a.MB * a_bytes, &mapU, bar_full + 8u * s, kb * kStageK,
+                      nb * a.BN, xi);
           if (++s == a.stages) { s = 0; ph ^= 1u; }
         }
         if (!ok) { *abort_p = 1u; break; }
@@ -249,12 +255,15 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
           if (!mbar_wait(bar_full + 8u * s, ph, abort_p)) { ok = false; break; }
           tc_fence_after();
           const uint32_t sa = base + (uint32_t)s * stage_bytes;
-          const uint64_t da = make_desc_sw128(sa), db = make_desc_sw128(sa + a_bytes);
+          const uint64_t db = make_desc_sw128(sa + (uint32_t)a.MB * a_bytes);
           const int remc = p.C - kb * kStageK;
           const int ksteps = remc >= kStageK ? 4 : (remc + 31) / 32;
-          for (int k = 0; k < ksteps; ++k)
-            mma_i8(tacc, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc,
-                   (kb | k) != 0 ? 1u : 0u);
+          for (int j = 0; j < a.MB; ++j) {
+            const uint64_t da = make_desc_sw128(sa + (uint32_t)j * a_bytes);
+            for (int k = 0; k < ksteps; ++k)
+              mma_i8(tacc + (uint32_t)(j * a.BN), da + (uint64_t)(k * 2), db + (uint64_t)(k * 2),
+                     idesc, (kb | k) != 0 ? 1u : 0u);
+          }
           mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
           if (++s == a.stages) { s = 0; ph ^= 1u; }
         }
@@ -293,15 +302,24 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
 TcGeom tc_geometry(const Params& p, int num_sms) {
   TcGeom g;
   g.BN = p.K >= 256 ? 256 : (p.K + 15) / 16 * 16;
-  const size_t per_stage = (size_t)kBM * kStageK + (size_t)g.BN * kStageK;
+  // narrow layers: several m-blocks share one U_q tile and one 256-column accumulator
+  g.MB = (g.BN == 64 || g.BN == 128) ? 256 / g.BN : 1;
+  const int n_mblk = (p.T + kBM - 1) / kBM;
+  // ... as long as that leaves every CTA at least three items to pipeline
+  const int n_nblk0 = (p.K + g.BN - 1) / g.BN;
+  while (g.MB > 1 && (p.t * p.t) * ((n_mblk + g.MB - 1) / g.MB) * n_nblk0 < 3 * num_sms) g.MB /= 2;
+  const size_t per_stage = (size_t)g.MB * kBM * kStageK + (size_t)g.BN * kStageK;
   g.stages = (int)((196 * 1024) / per_stage);
+  const int KB = (p.C + kStageK - 1) / kStageK;
+  if (g.stages > 2 * KB) g.stages = 2 * KB;   // two items' worth is all the ring can use
   if (g.stages > 8) g.stages = 8;
   if (g.stages < 1) g.stages = 1;
   int acc_stride = 32;
-  while (acc_stride < g.BN) acc_stride *= 2;
+  while (acc_stride < g.MB * g.BN) acc_stride *= 2;
   g.tmem_cols = 2 * acc_stride;
   g.smem = 1024 + g.stages * per_stage + 16 * g.stages + 64;
-  const int items = (p.t * p.t) * ((p.T + kBM - 1) / kBM) * ((p.K + g.BN - 1) / g.BN);
+  const int n_mgrp = (n_mblk + g.MB - 1) / g.MB;
+  const int items = (p.t * p.t) * n_mgrp * ((p.K + g.BN - 1) / g.BN);
   g.grid = items < num_sms ? items : num_sms;
   return g;
 }
@@ -319,7 +337,8 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
   GemmTcArgs a;
   a.BN = g.BN; a.stages = g.stages; a.tmem_cols = g.tmem_cols; a.acc_stride = g.tmem_cols / 2;
   a.out_mode = out_mode;
-  a.n_mblk = (p.T + kBM - 1) / kBM;
+  a.MB = g.MB;
+  a.n_mblk = ((p.T + kBM - 1) / kBM + g.MB - 1) / g.MB;
   a.n_nblk = (p.K + g.BN - 1) / g.BN;
   a.n_items = p.t * p.t * a.n_mblk * a.n_nblk;
   return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,

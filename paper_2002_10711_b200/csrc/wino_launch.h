@@ -35,7 +35,7 @@ int launch_output_transform_tma(const Params& p, const LaunchOpt& o, const CUten
                                 const CUtensorMap& mapY, const float* bias, float s_Y, int* status,
                                 cudaStream_t st);
 
-struct TcGeom { int BN, stages, tmem_cols, grid; size_t smem; };
+struct TcGeom { int BN, MB, stages, tmem_cols, grid; size_t smem; };
 TcGeom tc_geometry(const Params& p, int num_sms);
 int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,
                    const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
