@@ -22,8 +22,9 @@
  *   bias float [K]               in real units (optional)
  *
  * Arithmetic contract (what "the same result" means, bit for bit):
- *   - quantizer  Q(v; mult, z, qmin, qmax) = clamp(rne(v * mult) + z, qmin, qmax)
- *     with one fp32 multiply, round-half-to-even, and mult a precomputed fp32:
+ *   - quantizer  Q(v; mult, z, qmin, qmax) = clamp(rne(v * mult) + z, qmin, qmax):
+ *     the exact product of the fp32 value v and the fp32 multiplier is rounded
+ *     once, half to even; mult is precomputed,
  *     mult = (float)((double)s_src / (double)s_dst);
  *   - a transform  Z = (L X) L^T  is evaluated as a left pass then a right pass,
  *     each entry one fused-multiply-add chain starting from 0.0f and running

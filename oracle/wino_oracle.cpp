@@ -141,13 +141,15 @@ void cook_toom_rat(int m, const Rat* pts, std::vector<Rat>& BT, std::vector<Rat>
 }
 
 // ---------------------------------------------------------------------------
-// Uniform quantizer (Section 5.1: per-layer symmetric uniform quantization;
-// rounding to nearest-even, clamp, fixed multiplier).
+// Uniform quantizer (Section 5.1: per-layer symmetric uniform quantization):
+// code = clamp(round_half_even(v * mult) + z), the rounding applied to the exact
+// product of the fp32 value and the fixed fp32 multiplier.
 // ---------------------------------------------------------------------------
 inline int32_t quantize(float v, float mult, int32_t z, int32_t qmin, int32_t qmax) {
-  float scaled = v * mult;                 // one fp32 rounding
-  float r = std::nearbyintf(scaled);       // ties to even (default rounding mode)
-  float lo = (float)(qmin - z), hi = (float)(qmax - z);
+  // the product of two binary32 numbers is exact in binary64, so this rounds the
+  // exact real product once, ties to even (default rounding mode)
+  double r = std::nearbyint((double)v * (double)mult);
+  double lo = (double)(qmin - z), hi = (double)(qmax - z);
   if (r < lo) r = lo;
   if (r > hi) r = hi;
   return (int32_t)r + z;

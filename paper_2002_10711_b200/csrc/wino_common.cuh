@@ -30,14 +30,15 @@ struct Params {
 constexpr float kMagic = 12582912.0f;
 constexpr int kMagicBits = 0x4B400000;
 
-// Quantizer core: one fp32 multiply, clamp, round half to even.  Returns the
-// float kMagic + code; low byte of its bit pattern is the two's-complement code.
-// Clamping before rounding equals rounding before clamping because the bounds
-// are integers and rounding is monotone.
+// Quantizer core: round_half_even(v * mult) of the exact product, then clamp.
+// fmaf(v, mult, kMagic) rounds the exact value v*mult + kMagic once; for
+// |v*mult| < 2^22 the result lies in [2^23, 2^24) where floats are the integers,
+// so it equals kMagic + round_half_even(v*mult) (kMagic is even: ties agree).
+// Larger products stay monotone and are caught by the clamp.  Returns
+// kMagic + code; the low byte of the bit pattern is the two's-complement code.
 __device__ __forceinline__ float quant_magic(float v, float mult, float lo, float hi) {
-  float s = __fmul_rn(v, mult);
-  s = fminf(fmaxf(s, lo), hi);
-  return __fadd_rn(s, kMagic);
+  const float r = __fmaf_rn(v, mult, kMagic);
+  return fminf(fmaxf(r, __fadd_rn(lo, kMagic)), __fadd_rn(hi, kMagic));
 }
 __device__ __forceinline__ int magic_to_int(float r) { return __float_as_int(r) - kMagicBits; }
 __device__ __forceinline__ float magic_to_float(float r) { return __fsub_rn(r, kMagic); }

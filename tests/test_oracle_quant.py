@@ -2,6 +2,7 @@
 uniform quantization; round-half-to-even, clamp)."""
 import json
 import os
+from fractions import Fraction
 
 import numpy as np
 
@@ -18,16 +19,27 @@ def test_rounding_table():
 
 
 def test_against_second_implementation():
-    # independent statement: numpy's rint on the fp32 product, integer clamp afterwards
+    # independent statement: numpy's rint on the exact (float64) product of the two
+    # float32 numbers, integer clamp afterwards
     n = 20000
     v = (wi.normal(7, 1, n) * 300).astype(np.float32)
     v[:200] = (np.arange(200) - 100).astype(np.float32) / 2  # exact ties
     mult = np.float32(0.37)
     for z, qmin, qmax in ((0, -127, 127), (3, -127, 127), (0, 0, 127), (-10, -128, 127)):
-        prod = (v * mult).astype(np.float32)
+        prod = v.astype(np.float64) * np.float64(mult)
         want = np.clip(np.rint(prod).astype(np.int64) + z, qmin, qmax)
         got = np.array([oracle.quantize(x, mult, z, qmin, qmax) for x in v])
         assert (got == want).all()
+
+
+def test_product_is_rounded_once_not_twice():
+    # a product that the fp32 multiply would round onto a tie: v * mult = 2.5 + 2^-25
+    # exactly; rounding it to fp32 first gives 2.5 -> 2, rounding the exact value gives 3
+    v, mult = np.float32(1.25 * (1 + 2.0 ** -23)), np.float32(2.0 * (1 - 2.0 ** -24))
+    exact = Fraction(float(v)) * Fraction(float(mult))
+    assert exact > Fraction(5, 2) and np.float32(v * mult) == np.float32(2.5)
+    assert oracle.quantize(v, mult) == 3
+    assert oracle.quantize(-v, mult) == -3
 
 
 def test_multipliers_are_single_rounded_double_ratios():
