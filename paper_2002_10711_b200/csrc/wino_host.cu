@@ -53,7 +53,7 @@ struct wino_plan {
   mutable const void* map_uq_ptr;
   mutable CUtensorMap mapV, mapU;
   // maps of the TMA-staged transform kernels, keyed by buffer address
-  mutable MapCache cache_x, cache_vst, cache_mld, cache_y;
+  mutable MapCache cache_x, cache_vst, cache_mld, cache_y, cache_uf;
   // last forward call, for wino_debug_dump_stage
   mutable const int8_t* last_uq;
   mutable void* last_ws;
@@ -136,6 +136,7 @@ bool path_supported(const wino_plan_t* pl, int path) {
     case WINO_PATH_STAGED_TC_PTR: return C % 16 == 0 && K % 16 == 0;
     case WINO_PATH_STAGED_DP4A: return C % 4 == 0 && K % 4 == 0;
     case WINO_PATH_SMALLC: return C % 4 == 0 && K % 4 == 0 && C <= 32 && K <= 32;
+    case WINO_PATH_FUSED_F2: return fused_f2_supported(pl->p, pl->std_mats);
     default: return false;
   }
 }
@@ -217,6 +218,20 @@ const CUtensorMap* map_stage(const wino_plan_t* pl, MapCache& cache, const void*
   return m;
 }
 
+// U_q for the fused F2 kernel: [16][K][C], box {64, 64, 1}, 64-byte swizzle
+const CUtensorMap* map_u_fused(const wino_plan_t* pl, const void* Uq) {
+  if (const CUtensorMap* m = pl->cache_uf.find(Uq)) return m;
+  const Params& p = pl->p;
+  const uint64_t dims[3] = {(uint64_t)p.C, (uint64_t)p.K, 16};
+  const uint32_t box[3] = {64, 64, 1};
+  CUtensorMap* m = pl->cache_uf.slot(Uq);
+  if (encode_tiled(m, Uq, 3, dims, box, CU_TENSOR_MAP_SWIZZLE_64B) != WINO_OK) {
+    pl->cache_uf.key[(pl->cache_uf.next + MapCache::kN - 1) % MapCache::kN] = nullptr;
+    return nullptr;
+  }
+  return m;
+}
+
 int launch_gemm(const wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void* out, int out_mode,
                 unsigned* absmaxM, bool pdl, cudaStream_t st) {
   const Params& p = pl->p;
@@ -249,6 +264,13 @@ int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const
     pl->launches++;
     return launch_smallc(pl->p, opt_of(pl, pdl), x, Uq, bias, y, pl->s_Y, st);
   }
+  if (pl->path == WINO_PATH_FUSED_F2 && !calib && stage_mask == 7) {
+    const CUtensorMap* mu = map_u_fused(pl, Uq);
+    if (mu == nullptr) return WINO_ERR_CUDA;
+    pl->launches++;
+    return launch_fused_f2(pl->p, opt_of(pl, pdl), *mu, x, bias, y, pl->s_Y, pl->num_sms,
+                           pl->status_dev, st);
+  }
   if (ws == nullptr) return WINO_ERR_WORKSPACE;
   if (!aligned16(ws)) return WINO_ERR_ALIGNMENT;
   int8_t* Vq = reinterpret_cast<int8_t*>(ws);
@@ -256,9 +278,9 @@ int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const
   // calibration on a small-channel plan uses the dp4a kernel for the middle stage
   wino_plan_t tmp_holder;
   const wino_plan_t* run = pl;
-  if (pl->path == WINO_PATH_SMALLC) {
+  if (pl->path == WINO_PATH_SMALLC || pl->path == WINO_PATH_FUSED_F2) {
     tmp_holder = *pl;
-    tmp_holder.path = WINO_PATH_STAGED_DP4A;
+    tmp_holder.path = pl->path == WINO_PATH_SMALLC ? WINO_PATH_STAGED_DP4A : WINO_PATH_STAGED_TC_PTR;
     run = &tmp_holder;
   }
   const bool ev = pl->stage_ev_on;
@@ -366,6 +388,7 @@ int wino_plan(const wino_desc_t* desc, wino_plan_t** out) {
   pl->std_mats = d.m == 2 ? is_std<2>(p.BT, p.AT) : d.m == 4 ? is_std<4>(p.BT, p.AT)
                                                                : is_std<6>(p.BT, p.AT);
   if (path_supported(pl, WINO_PATH_SMALLC)) pl->path = WINO_PATH_SMALLC;
+  else if (path_supported(pl, WINO_PATH_FUSED_F2)) pl->path = WINO_PATH_FUSED_F2;
   else if (path_supported(pl, WINO_PATH_STAGED_TC)) pl->path = WINO_PATH_STAGED_TC;
   else if (path_supported(pl, WINO_PATH_STAGED_DP4A)) pl->path = WINO_PATH_STAGED_DP4A;
   else { delete pl; return WINO_ERR_UNSUPPORTED; }
@@ -402,7 +425,7 @@ int wino_plan_path(const wino_plan_t* pl) { return pl ? pl->path : WINO_ERR_INVA
 
 int wino_plan_force_path(wino_plan_t* pl, int path) {
   if (pl == nullptr) return WINO_ERR_INVALID;
-  if (path < WINO_PATH_STAGED_TC || path > WINO_PATH_STAGED_TC_PTR) return WINO_ERR_INVALID;
+  if (path < WINO_PATH_STAGED_TC || path > WINO_PATH_FUSED_F2) return WINO_ERR_INVALID;
   if (!path_supported(pl, path)) return WINO_ERR_UNSUPPORTED;
   pl->path = path;
   return WINO_OK;
@@ -457,7 +480,8 @@ int wino_debug_run_stages(const wino_plan_t* pl, int stage_mask, const int8_t* x
                           const float* bias, void* y, void* ws, void* stream) {
   if (pl == nullptr || x == nullptr || Uq == nullptr || y == nullptr) return WINO_ERR_INVALID;
   if (stage_mask < 1 || stage_mask > 7) return WINO_ERR_INVALID;
-  if (pl->path == WINO_PATH_SMALLC) return WINO_ERR_UNSUPPORTED;
+  if ((pl->path == WINO_PATH_SMALLC || pl->path == WINO_PATH_FUSED_F2) && stage_mask != 7)
+    return WINO_ERR_UNSUPPORTED;   // the fused paths have no separate stages
   if (!aligned16(x) || !aligned16(Uq) || !aligned16(y) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
   return forward_impl(pl, x, Uq, bias, y, ws, nullptr, (cudaStream_t)stream, stage_mask);

@@ -43,6 +43,12 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
 int launch_smallc(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
                   const float* bias, void* y, float s_Y, cudaStream_t st);
 
+// Fully fused F2 kernel for narrow layers (C in {32, 64}, K <= 64, Cook-Toom matrices).
+bool fused_f2_supported(const Params& p, bool std_mats);
+int launch_fused_f2(const Params& p, const LaunchOpt& o, const CUtensorMap& mapU, const int8_t* x,
+                    const float* bias, void* y, float s_Y, int num_sms, int* status,
+                    cudaStream_t st);
+
 enum { kOutMq = 0, kOutI32 = 1 };
 constexpr int kBM = 128;      // tiles per GEMM block (MMA M)
 constexpr int kStageK = 128;  // channels (bytes) per shared-memory stage

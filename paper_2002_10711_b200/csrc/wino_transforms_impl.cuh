@@ -18,139 +18,12 @@
 #pragma once
 #include <cstdlib>
 #include "wino_launch.h"
+#include "wino_transform_math.cuh"
 
 #define WINO_CAT_(a, b) a##b
 #define WINO_CAT(a, b) WINO_CAT_(a, b)
 
 namespace wino {
-
-enum { kDense = 0, kSparse = 1, kExact = 2 };
-
-template <int CPT> struct Pack;
-template <> struct Pack<1> { typedef uint8_t type; };
-template <> struct Pack<2> { typedef uint16_t type; };
-template <> struct Pack<4> { typedef uint32_t type; };
-
-__device__ __forceinline__ uint32_t insert_byte(uint32_t word, uint32_t bits, int ch) {
-  const uint32_t sel = ch == 0 ? 0x3214u : ch == 1 ? 0x3240u : ch == 2 ? 0x3410u : 0x4210u;
-  return __byte_perm(word, bits, sel);
-}
-
-// 1-D B^T for F4, factored (exact mode only).
-__device__ __forceinline__ void bt4_exact(const float (&d)[6], float (&r)[6]) {
-  const float t1 = __fsub_rn(d[3], d[1]);
-  const float t2 = __fsub_rn(d[4], d[2]);
-  const float u = __fmaf_rn(4.0f, d[2], -d[4]);
-  const float v = __fmaf_rn(4.0f, d[1], -d[3]);
-  r[0] = __fmaf_rn(4.0f, d[0], __fmaf_rn(-5.0f, d[2], d[4]));
-  r[1] = __fadd_rn(u, v);
-  r[2] = __fsub_rn(u, v);
-  r[3] = __fmaf_rn(2.0f, t1, t2);
-  r[4] = __fmaf_rn(-2.0f, t1, t2);
-  r[5] = __fmaf_rn(4.0f, d[1], __fmaf_rn(-5.0f, d[3], d[5]));
-}
-// 1-D A^T for F4, factored (exact mode only).
-__device__ __forceinline__ void at4_exact(const float (&m)[6], float (&y)[4]) {
-  const float a = __fadd_rn(m[1], m[2]);
-  const float b = __fsub_rn(m[1], m[2]);
-  const float c = __fadd_rn(m[3], m[4]);
-  const float d = __fsub_rn(m[3], m[4]);
-  y[0] = __fadd_rn(__fadd_rn(m[0], a), c);
-  y[1] = __fmaf_rn(2.0f, d, b);
-  y[2] = __fmaf_rn(4.0f, c, a);
-  y[3] = __fadd_rn(__fmaf_rn(8.0f, d, b), m[5]);
-}
-
-// V = (B^T d) B for one channel.  d is given column-wise through `col(l, out)`.
-template <int M, int MODE, typename ColFn>
-__device__ __forceinline__ void input_transform_2d(const Params& p, ColFn col,
-                                                   float (&V)[(M + 2) * (M + 2)]) {
-  constexpr int T_ = M + 2;
-  constexpr bool STD = MODE != kDense;
-  using MT = Mat<M, STD>;
-  float P[T_][T_];
-#pragma unroll
-  for (int l = 0; l < T_; ++l) {
-    float dcol[T_];
-    col(l, dcol);
-    if constexpr (MODE == kExact && M == 4) {
-      float r[6];
-      bt4_exact(dcol, r);
-#pragma unroll
-      for (int i = 0; i < T_; ++i) P[i][l] = r[i];
-    } else {
-#pragma unroll
-      for (int i = 0; i < T_; ++i) {
-        float acc = 0.0f;
-#pragma unroll
-        for (int k = 0; k < T_; ++k) acc = chain<STD>(MT::bt(p, i, k), dcol[k], acc);
-        P[i][l] = acc;
-      }
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < T_; ++i) {
-    if constexpr (MODE == kExact && M == 4) {
-      float r[6];
-      bt4_exact(P[i], r);
-#pragma unroll
-      for (int j = 0; j < T_; ++j) V[i * T_ + j] = r[j];
-    } else {
-#pragma unroll
-      for (int j = 0; j < T_; ++j) {
-        float acc = 0.0f;
-#pragma unroll
-        for (int l = 0; l < T_; ++l) acc = chain<STD>(MT::bt(p, j, l), P[i][l], acc);
-        V[i * T_ + j] = acc;
-      }
-    }
-  }
-}
-
-// Y = A^T (m A) for one channel: right factor first.  m row-wise via `row(i, out)`.
-template <int M, int MODE, typename RowFn>
-__device__ __forceinline__ void output_transform_2d(const Params& p, RowFn row,
-                                                    float (&Y)[M * M]) {
-  constexpr int T_ = M + 2;
-  constexpr bool STD = MODE != kDense;
-  using MT = Mat<M, STD>;
-  float R[T_][M];
-#pragma unroll
-  for (int i = 0; i < T_; ++i) {
-    float mrow[T_];
-    row(i, mrow);
-    if constexpr (MODE == kExact && M == 4) {
-      at4_exact(mrow, R[i]);
-    } else {
-#pragma unroll
-      for (int jp = 0; jp < M; ++jp) {
-        float acc = 0.0f;
-#pragma unroll
-        for (int j = 0; j < T_; ++j) acc = chain<STD>(MT::at(p, jp, j), mrow[j], acc);
-        R[i][jp] = acc;
-      }
-    }
-  }
-#pragma unroll
-  for (int jp = 0; jp < M; ++jp) {
-    if constexpr (MODE == kExact && M == 4) {
-      float c[6], y4[4];
-#pragma unroll
-      for (int i = 0; i < T_; ++i) c[i] = R[i][jp];
-      at4_exact(c, y4);
-#pragma unroll
-      for (int ip = 0; ip < M; ++ip) Y[ip * M + jp] = y4[ip];
-    } else {
-#pragma unroll
-      for (int ip = 0; ip < M; ++ip) {
-        float acc = 0.0f;
-#pragma unroll
-        for (int i = 0; i < T_; ++i) acc = chain<STD>(MT::at(p, ip, i), R[i][jp], acc);
-        Y[ip * M + jp] = acc;
-      }
-    }
-  }
-}
 
 // ---------------------------------------------------------------------------
 // Stage 2: filters.  w [K][3][3][C] int8 -> U_q [t*t][K][C] int8.

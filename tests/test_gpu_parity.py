@@ -11,7 +11,7 @@ from helpers import build_layer, small
 
 pytestmark = pytest.mark.gpu
 
-TC, DP4A, SMALLC, TC_PTR = 1, 2, 3, 4
+TC, DP4A, SMALLC, TC_PTR, FUSED = 1, 2, 3, 4, 5
 
 
 def _compare(L, x_q, w_q, bias, path, dumps=True):
@@ -99,6 +99,58 @@ def test_small_channel_path(m, shape):
     _compare(L, x_q, w_q, bias, DP4A, dumps=True)
 
 
+FUSED_SHAPES = [
+    # N, C, H, W, K
+    (2, 64, 8, 8, 64),
+    (1, 32, 7, 9, 48),        # ragged tiles; K = 48: second 32-channel block half empty
+    (3, 64, 13, 5, 16),
+    (1, 32, 32, 32, 32),
+    (40, 64, 32, 32, 64),     # 10240 tiles = 80 blocks of 128
+    (100, 64, 30, 30, 64),    # 22500 tiles: more blocks than SMs, last block partial
+]
+
+
+@pytest.mark.parametrize("shape", FUSED_SHAPES)
+def test_fused_f2_kernel(shape):
+    N, C, H, W, K = shape
+    wl = wi.Workload("fu", 3500 + C + K, N, C, H, W, K, 2)
+    L, x_q, w_q, bias = build_layer(wl)
+    from paper_2002_10711_b200 import binding
+    if C > 32 or K > 32:                                   # else the warp-shuffle path is chosen
+        assert binding.Plan.from_layer(L).path == FUSED
+    _compare(L, x_q, w_q, bias, FUSED, dumps=False)
+
+
+@pytest.mark.parametrize("variant", ["no_qm", "float_out", "no_qm_float", "relu", "no_bias", "zero_points"])
+def test_fused_f2_variants(variant):
+    wl = wi.Workload("fv", 3600, 3, 64, 10, 12, 64, 2)
+    kw = {}
+    if variant in ("no_qm", "no_qm_float"):
+        kw["q_M"] = False
+    if variant in ("float_out", "no_qm_float"):
+        kw["out_dtype"] = 1
+    if variant == "relu":
+        kw["relu"] = True
+    if variant == "no_bias":
+        kw["with_bias"] = False
+    L, x_q, w_q, bias = build_layer(wl, **kw)
+    if variant == "zero_points":
+        L.q_x.zero_point = 5
+        L.q_w.zero_point = -3
+        L.q_Y.zero_point = 7
+    _compare(L, x_q, w_q, bias, FUSED, dumps=False)
+
+
+def test_fused_f2_refuses_other_shapes():
+    from paper_2002_10711_b200 import binding
+    for m, C, K, flex in ((4, 64, 64, False), (2, 128, 64, False), (2, 64, 128, False), (2, 64, 64, True)):
+        wl = wi.Workload("fr", 3700, 1, C, 8, 8, K, m, flex=flex)
+        L, x_q, w_q, bias = build_layer(wl)
+        with pytest.raises(binding.WinoError) as e:
+            binding.Plan.from_layer(L, path=FUSED)
+        assert e.value.code == binding.ERR_UNSUPPORTED
+
+
 def test_saturating_scales_clip_identically():
     wl = wi.Workload("sat", 3400, 2, 32, 8, 8, 32, 4)
     L, x_q, w_q, bias = build_layer(wl)
@@ -123,6 +175,8 @@ def test_full_size_configs(name):
     g = _compare(L, x_q, w_q, bias, TC)
     assert g["launches"] >= 4
     _compare(L, x_q, w_q, bias, TC_PTR)
+    if name == "cfg2":
+        _compare(L, x_q, w_q, bias, FUSED, dumps=False)
 
 
 def test_cfg3_without_qm():
