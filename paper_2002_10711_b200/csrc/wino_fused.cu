@@ -63,8 +63,8 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
   const uint32_t sBias = sB + 16u * kBTile;         // 64 floats: bias / s_Y
   const uint32_t bar_b = sBias + 256u;              // U_q landed
   const uint32_t bar_a_full = bar_b + 8u;           // workers -> control: A tiles written
-  const uint32_t bar_acc = bar_a_full + 8u;         // control -> workers: accumulators complete
-  const uint32_t bar_tmem_free = bar_acc + 8u;      // workers -> control: accumulators drained
+  const uint32_t bar_acc = bar_a_full + 8u;         // control -> workers: 4 barriers, one per row of positions
+  const uint32_t bar_tmem_free = bar_acc + 32u;     // workers -> control: accumulators drained
   const uint32_t tmem_slot = bar_tmem_free + 8u;
   const uint32_t abort_slot = tmem_slot + 4u;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
@@ -80,7 +80,7 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
   if (threadIdx.x == 0) {
     mbar_init(bar_b, 1);
     mbar_init(bar_a_full, kFusedWorkers);
-    mbar_init(bar_acc, 1);
+    for (int i = 0; i < 4; ++i) mbar_init(bar_acc + 8u * i, 1);
     mbar_init(bar_tmem_free, kFusedWorkers);
     *abort_p = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -113,8 +113,10 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
             for (int k = 0; k < ksteps; ++k)
               mma_i8(tmem_base + (uint32_t)(xi * 32), da + (uint64_t)(k * 2), db + (uint64_t)(k * 2),
                      idesc, k != 0 ? 1u : 0u);
+            // a row of four positions is complete: its epilogue may start while the
+            // remaining rows are still being multiplied
+            if ((xi & 3) == 3) mma_commit(bar_acc + 8u * (uint32_t)(xi >> 2));
           }
-          mma_commit(bar_acc);
         }
       }
       if (!ok) *abort_p = 1u;
@@ -139,47 +141,69 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
       // the MMAs of the previous block must be done reading the A tiles
       // (implied: its last accumulator round was observed complete below)
       // ---- input transform: A tiles for all 16 positions ----
+      // loads of the next task are issued before the current one is transformed
+      auto load_task = [&](int task, uint32_t (&wd)[16]) {
+        const int c4 = task % C4, tau = mb * 128 + task / C4;
+        if (task >= tasks || tau >= p.T) {
+#pragma unroll
+          for (int i = 0; i < 16; ++i) wd[i] = zword;
+          return;
+        }
+        const int tw = tau % p.TW;
+        const int th = (tau / p.TW) % p.TH;
+        const int n = tau / (p.TW * p.TH);
+        // one 64-bit base; row / column offsets are 32-bit, coordinates clamped
+        // into the image and validity applied as a mask afterwards
+        const uint32_t* xb = x32 + (long)n * p.H * p.W * C4 + c4;
+        int roff[4], coff[4];
+        uint32_t rmask[4], cmask[4];
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+          const int h = th * 2 - 1 + a, wv = tw * 2 - 1 + a;
+          rmask[a] = (h >= 0 && h < p.H) ? 0xFFFFFFFFu : 0u;
+          cmask[a] = (wv >= 0 && wv < p.W) ? 0xFFFFFFFFu : 0u;
+          roff[a] = min(max(h, 0), p.H - 1) * p.W * C4;
+          coff[a] = min(max(wv, 0), p.W - 1) * C4;
+        }
+#pragma unroll
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int b = 0; b < 4; ++b) {
+            const uint32_t v = __ldg(xb + (roff[a] + coff[b])) ^ 0x80808080u;
+            const uint32_t mk = rmask[a] & cmask[b];
+            wd[a * 4 + b] = (v & mk) | (zword & ~mk);
+          }
+      };
+      uint32_t wd[16];
+      load_task(wid, wd);
       for (int task = wid; task < tasks; task += 32 * kFusedWorkers) {
         const int c4 = task % C4, tl = task / C4;
-        const int tau = mb * 128 + tl;
+        uint32_t wn[16];
+        load_task(task + 32 * kFusedWorkers, wn);
         uint32_t out[16];
 #pragma unroll
         for (int i = 0; i < 16; ++i) out[i] = 0u;
-        if (tau < p.T) {
-          const int tw = tau % p.TW;
-          const int th = (tau / p.TW) % p.TH;
-          const int n = tau / (p.TW * p.TH);
-          uint32_t wd[16];
-#pragma unroll
-          for (int a = 0; a < 4; ++a) {
-            const int h = th * 2 - 1 + a;
-#pragma unroll
-            for (int b = 0; b < 4; ++b) {
-              const int wv = tw * 2 - 1 + b;
-              const bool in = h >= 0 && h < p.H && wv >= 0 && wv < p.W;
-              wd[a * 4 + b] =
-                  in ? (__ldg(x32 + (((long)n * p.H + h) * p.W + wv) * C4 + c4) ^ 0x80808080u) : zword;
-            }
-          }
+        // tiles past the end carry zero patches; their rows are never stored
 #pragma unroll 1
-          for (int ch = 0; ch < 4; ++ch) {
-            const uint32_t sel_in = 0x7440u | (uint32_t)ch;
-            const uint32_t sel_out = insert_selector(ch);
-            float V[16];
-            input_transform_2d<2, kSparse>(p, [&](int l, float (&dcol)[4]) {
+        for (int ch = 0; ch < 4; ++ch) {
+          const uint32_t sel_in = 0x7440u | (uint32_t)ch;
+          const uint32_t sel_out = insert_selector(ch);
+          float V[16];
+          input_transform_2d<2, kSparse>(p, [&](int l, float (&dcol)[4]) {
 #pragma unroll
-              for (int a = 0; a < 4; ++a) dcol[a] = byte_to_float_sel(wd[a * 4 + l], sel_in, ubias);
-            }, V);
+            for (int a = 0; a < 4; ++a) dcol[a] = byte_to_float_sel(wd[a * 4 + l], sel_in, ubias);
+          }, V);
 #pragma unroll
-            for (int xi = 0; xi < 16; ++xi) {
-              const float r = quant_magic(V[xi], p.mult_V, p.lo_V, p.hi_V);
-              out[xi] = __byte_perm(out[xi], __float_as_uint(r), sel_out);
-            }
+          for (int xi = 0; xi < 16; ++xi) {
+            const float r = quant_magic(V[xi], p.mult_V, p.lo_V, p.hi_V);
+            out[xi] = __byte_perm(out[xi], __float_as_uint(r), sel_out);
           }
         }
         const uint32_t off = sw64_offset(tl, c4 * 4);
 #pragma unroll
         for (int xi = 0; xi < 16; ++xi) sts32(sA + (uint32_t)xi * kATile + off, out[xi]);
+#pragma unroll
+        for (int i = 0; i < 16; ++i) wd[i] = wn[i];
       }
       fence_async_smem();      // generic-proxy writes -> visible to the tensor core's async reads
       __syncwarp();
@@ -191,9 +215,18 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
       const int tw = tau % p.TW;
       const int th = (tau / p.TW) % p.TH;
       const int n = tau / (p.TW * p.TH);
+      const long obase = (((long)n * p.H + th * 2) * p.W + tw * 2) * p.K;   // pixel (0,0) of the tile
       for (int nb = 0; nb < n_nblk; ++nb, ++round) {
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_acc, round & 1u, abort_p))) { ok = false; break; }
-        tc_fence_after();
+        // wait for a row of positions: lane 0 polls (bounded), every lane then
+        // observes the completed phase once
+        auto wait_row = [&](int i) -> bool {
+          int got = 1;
+          if (lane == 0) got = mbar_wait(bar_acc + 8u * (uint32_t)i, round & 1u, abort_p) ? 1 : 0;
+          if (__shfl_sync(0xffffffffu, got, 0) == 0) return false;
+          (void)mbar_try_wait(bar_acc + 8u * (uint32_t)i, round & 1u);
+          tc_fence_after();
+          return true;
+        };
         const uint32_t tlane = tmem_base + ((uint32_t)(quad * 32) << 16);
 #pragma unroll 1
         for (int half = 0; half < 2; ++half) {
@@ -201,6 +234,7 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
           float Y[2][2][4];
 #pragma unroll
           for (int i = 0; i < 4; ++i) {                        // row of positions (i, 0..3)
+            if (half == 0 && !wait_row(i)) { ok = false; break; }
             uint32_t acc[4][4];
 #pragma unroll
             for (int j = 0; j < 4; ++j)
@@ -211,7 +245,8 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
               float mrow[4];
 #pragma unroll
               for (int j = 0; j < 4; ++j) {
-                const float f = __int2float_rn((int)acc[j][q]);
+                // |M| <= 127^2 * 64 < 2^22: exact conversion by one add and one subtract
+                const float f = small_int_to_float((int)acc[j][q]);
                 mrow[j] = p.qM_enabled ? magic_to_float(quant_magic(f, p.mult_M, p.lo_M, p.hi_M)) : f;
               }
               // R = m A (right factor first): chains over j with A^T rows (1,1,1,0), (0,1,-1,1)
@@ -231,6 +266,7 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
               }
             }
           }
+          if (!ok) break;
           if (row_ok && kc < p.K) {
 #pragma unroll
             for (int ip = 0; ip < 2; ++ip)
@@ -238,7 +274,7 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
               for (int jp = 0; jp < 2; ++jp) {
                 const int h = th * 2 + ip, wv = tw * 2 + jp;
                 if (h >= p.H || wv >= p.W) continue;
-                const long o = (((long)n * p.H + h) * p.W + wv) * p.K + kc;
+                const long o = obase + (long)((ip * p.W + jp) * p.K + kc);
                 if (p.out_dtype == 0) {
                   uint32_t word = 0u;
 #pragma unroll
@@ -258,6 +294,7 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
               }
           }
         }
+        if (!ok) break;
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tmem_free);
@@ -282,7 +319,7 @@ bool fused_f2_supported(const Params& p, bool std_mats) {
 int launch_fused_f2(const Params& p, const LaunchOpt& o, const CUtensorMap& mapU, const int8_t* x,
                     const float* bias, void* y, float s_Y, int num_sms, int* status,
                     cudaStream_t st) {
-  const size_t smem = 1024 + 16 * (size_t)kATile + 16 * (size_t)kBTile + 256 + 64;
+  const size_t smem = 1024 + 16 * (size_t)kATile + 16 * (size_t)kBTile + 256 + 128;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k_fused_f2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
