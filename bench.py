@@ -236,7 +236,8 @@ def run_ours(args, wl):
             for i in range(chunk):
                 step(i)
     torch.cuda.synchronize()
-    launches_per_step = 3 if plan.path != binding.PATH_SMALLC else 1
+    single_kernel = plan.path in (binding.PATH_SMALLC, binding.PATH_FUSED_F2)
+    launches_per_step = 1 if single_kernel else 3
     graph.replay()
     torch.cuda.synchronize()
 
@@ -273,7 +274,15 @@ def run_ours(args, wl):
     peaks = load_peaks()
     roofline = None
     stages = None
-    if plan.path != binding.PATH_SMALLC:
+    if single_kernel:
+        # one fused kernel per step: its launch duration is the step time
+        alg_bytes = xb + yb + plan.weight_bytes
+        ach = alg_bytes / (ms_local / args.steps * 1e-3) / 1e9
+        roofline = {"kernel": "k_fused_f2" if plan.path == binding.PATH_FUSED_F2 else "k_smallc",
+                    "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                    "frac": ach / peaks["hbm_gbs"], "traffic": None,
+                    "peak_note": f"of {peaks['source']}"}
+    else:
         names = ["input_transform", "hadamard_gemm", "output_transform"]
         us = []
         for mask in (1, 2, 4):
@@ -403,7 +412,7 @@ def run_ours(args, wl):
             "config": workload_config(
                 wl, f"inputs rotate over {R} buffer sets ({R * (xb + yb + plan.weight_bytes) / 1e6:.0f} MB > L2)"),
             "wino_domain_TOPS": wino_ops(wl, wl.N) * world / (ms_per_step * 1e-3) / 1e12,
-            "path": {1: "staged_tc", 2: "staged_dp4a", 3: "smallc"}[plan.path],
+            "path": {1: "staged_tc", 2: "staged_dp4a", 3: "smallc", 4: "staged_tc_ptr", 5: "fused_f2"}[plan.path],
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "layer_roofline": layer_roof, "stages": stages,
             "weight_transform": {"us": wt_us, "GBps": wt_bytes / (wt_us * 1e-6) / 1e9,
