@@ -216,8 +216,8 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------
-// Launchers.  CC (or KC) is the largest of 256 / 128 / 64 that divides the
-// channel count; G makes the block at least 64 threads.
+// Launchers.  CC (or KC) is 128 when it divides the channel count (one tile per
+// block), else 64 (four tiles per block).
 // ---------------------------------------------------------------------------
 namespace {
 
@@ -250,16 +250,13 @@ int input_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapX, const CUt
                    int* status, cudaStream_t st) {
   const int cc = tma_chunk(p.C);
   if (tma_cpt((long)p.T * p.C) == 4)
-    return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 4>(p, pdl, mapX, mapV, status, st)
-         : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 4>(p, pdl, mapX, mapV, status, st)
+    return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 4>(p, pdl, mapX, mapV, status, st)
                      : input_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapX, mapV, status, st);
   if (tma_cpt((long)p.T * p.C) == 1)
-    return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 1>(p, pdl, mapX, mapV, status, st)
-         : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 1>(p, pdl, mapX, mapV, status, st)
+    return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 1>(p, pdl, mapX, mapV, status, st)
                      : input_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapX, mapV, status, st);
-  return cc == 256 ? input_tma_launch<M, MODE, 256, 1, 2>(p, pdl, mapX, mapV, status, st)
-       : cc == 128 ? input_tma_launch<M, MODE, 128, 2, 2>(p, pdl, mapX, mapV, status, st)
-                   : input_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapX, mapV, status, st);
+  return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 2>(p, pdl, mapX, mapV, status, st)
+                     : input_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapX, mapV, status, st);
 }
 
 template <int M, int MODE, int KC, int G, int CPT>
@@ -282,16 +279,13 @@ int output_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapM, const CU
                     const float* bias, float s_Y, int* status, cudaStream_t st) {
   const int kc = tma_chunk(p.K);
   if (tma_cpt((long)p.T * p.K) == 4)
-    return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+    return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
                      : output_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
   if (tma_cpt((long)p.T * p.K) == 1)
-    return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+    return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
                      : output_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st);
-  return kc == 256 ? output_tma_launch<M, MODE, 256, 1, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-       : kc == 128 ? output_tma_launch<M, MODE, 128, 2, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                   : output_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+  return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                     : output_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st);
 }
 
 }  // namespace
