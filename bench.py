@@ -33,9 +33,9 @@ if ROOT not in sys.path:
 
 import wino_inputs as wi  # noqa: E402
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture
-# summarised in profiles/cfg3_staged_tc_launches_and_kernels.md; valid for cfg3 and for the
-# kernels as profiled there (set an entry to None when its kernel changes).
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture
+# of the cfg3 workload with the kernels as they stand; set an entry to None when its kernel
+# changes and the counters have not been taken again.
 NCU_TRAFFIC_CFG3 = {"k_input_transform_tma": 4.21e6, "k_gemm_tc": 11.84e6,
                     "k_output_transform_tma": 9.45e6}
 
