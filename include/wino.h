@@ -46,6 +46,11 @@
  *
  * Errors.  Every function returns WINO_OK (0) or a negative code; nothing
  * throws, aborts or traps.  Launches are asynchronous on the given stream.
+ *
+ * Devices and threads.  A plan belongs to the device that was current when
+ * wino_plan ran (its status word lives there); use it with that device current.
+ * A plan is not thread-safe: calls on one plan must not overlap in time on the
+ * host.  Different plans may be used from different threads.
  */
 #ifndef WINO_H_
 #define WINO_H_
