@@ -149,7 +149,9 @@ def run_reference(args, wl):
 
 def workload_config(wl, l2_note):
     return {"workload": f"{wl.name}: ResNet-18 CIFAR layer N={wl.N} C=K={wl.C} H=W={wl.H} "
-                        f"F({wl.m}x{wl.m},3x3) int8, per-stage max-abs scales",
+                        f"F({wl.m}x{wl.m},3x3) int8, "
+                        + ("all stage scales fixed" if wl.fixed_scales is not None
+                           else "per-stage max-abs scales"),
             "N": wl.N, "C": wl.C, "K": wl.K, "H": wl.H, "W": wl.W, "m": wl.m, "l2": l2_note}
 
 
@@ -200,7 +202,10 @@ def run_ours(args, wl):
         return binding.Plan(wl.N, wl.C, wl.H, wl.W, wl.K, wl.m, BT, G, AT, q(s_x), q(s_w), q(s_V),
                             q(s_U), q(s_M), q(s_Y), out_dtype=0)
 
-    s_V, s_U, s_M, s_Y = calibrate(make_plan, x_q, w_q, bias, s_x, s_w, device=dev)
+    if wl.fixed_scales is not None:
+        s_V = s_U = s_M = s_Y = float(np.float32(wl.fixed_scales))
+    else:
+        s_V, s_U, s_M, s_Y = calibrate(make_plan, x_q, w_q, bias, s_x, s_w, device=dev)
     plan = make_plan(s_V, s_U, s_M, s_Y)
 
     # ---- device buffers: R rotating sets so that x, y and U_q come from HBM ----

@@ -98,9 +98,9 @@ typedef struct {
 
 /* Problem statement of one layer.  BT, G, AT are HOST pointers to row-major
  * fp32 matrices BT[t][t], G[t][3], AT[m][t]; they are copied by wino_plan.
- * transforms_exact = 1 is the caller's promise that BT and AT are the Cook-Toom
- * matrices for the standard points, whose products with integer codes are exact
- * in fp32 (the library may then reorder sums; results are unchanged).
+ * transforms_exact is advisory: the library itself recognises the Cook-Toom
+ * matrices for the standard points (bit-for-bit comparison) and only then uses
+ * kernels that rely on their products with integer codes being exact in fp32.
  * out_dtype: 0 = int8 codes, 1 = float real values.
  * Restrictions (WINO_ERR_UNSUPPORTED otherwise): m in {2, 4, 6};
  * zero_point == 0 for q_V, q_U, q_M; C <= 1040 (so that (float)M is exact). */
