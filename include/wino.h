@@ -77,7 +77,7 @@ enum {
   WINO_PATH_AUTO = 0,
   WINO_PATH_STAGED_TC = 1,   /* transform kernels (TMA-staged where the shape allows) + tcgen05 int8 GEMMs */
   WINO_PATH_STAGED_DP4A = 2, /* transform kernels + integer-dot-product GEMMs on the ALUs */
-  WINO_PATH_SMALLC = 3,      /* one fused warp-shuffle kernel, C <= 32 and K <= 32 */
+  WINO_PATH_SMALLC = 3,      /* one fused warp-shuffle kernel, C <= 32 and K <= 32 (never chosen automatically) */
   WINO_PATH_STAGED_TC_PTR = 4, /* as 1, but always the pointer-based transform kernels */
   WINO_PATH_FUSED_F2 = 5     /* one fused tcgen05 kernel: m = 2, Cook-Toom matrices, C in {32, 64}, K <= 64 */
 };

@@ -116,8 +116,7 @@ def test_fused_f2_kernel(shape):
     wl = wi.Workload("fu", 3500 + C + K, N, C, H, W, K, 2)
     L, x_q, w_q, bias = build_layer(wl)
     from paper_2002_10711_b200 import binding
-    if C > 32 or K > 32:                                   # else the warp-shuffle path is chosen
-        assert binding.Plan.from_layer(L).path == FUSED
+    assert binding.Plan.from_layer(L).path == FUSED      # the automatic choice for these shapes
     _compare(L, x_q, w_q, bias, FUSED, dumps=False)
 
 

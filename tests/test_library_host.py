@@ -50,8 +50,11 @@ def test_sizes_and_paths():
     assert p.T == 2 * 2 * 2
     assert p.workspace_bytes >= 36 * p.T * 64 * 2
     assert p.path == binding.PATH_STAGED_TC
-    assert _plan(C=16, K=16).path == binding.PATH_SMALLC
-    assert _plan(C=20, K=24).path == binding.PATH_SMALLC
+    assert _plan(C=16, K=16).path == binding.PATH_STAGED_TC
+    assert _plan(C=20, K=24).path == binding.PATH_STAGED_DP4A
+    p = _plan(C=20, K=24)
+    p.force_path(binding.PATH_SMALLC)
+    assert p.path == binding.PATH_SMALLC
     assert _plan(C=36, K=40).path == binding.PATH_STAGED_DP4A
     assert _plan(m=2, C=64, K=64).path == binding.PATH_FUSED_F2
     assert _plan(m=2, C=64, K=128).path == binding.PATH_STAGED_TC
