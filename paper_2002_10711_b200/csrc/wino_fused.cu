@@ -189,7 +189,7 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
           const uint32_t sel_in = 0x7440u | (uint32_t)ch;
           const uint32_t sel_out = insert_selector(ch);
           float V[16];
-          input_transform_2d<2, kSparse>(p, [&](int l, float (&dcol)[4]) {
+          input_transform_2d<2, kExact>(p, [&](int l, float (&dcol)[4]) {
 #pragma unroll
             for (int a = 0; a < 4; ++a) dcol[a] = byte_to_float_sel(wd[a * 4 + l], sel_in, ubias);
           }, V);

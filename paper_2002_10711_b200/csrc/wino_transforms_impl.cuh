@@ -307,10 +307,8 @@ template <int M>
 int input_m(const Params& p, const LaunchOpt& o, const int8_t* x, int8_t* Vq, unsigned* absmax,
             cudaStream_t st) {
   if (!o.std_mats) return input_mode<M, kDense>(p, o.pdl, x, Vq, absmax, st);
-  // Cook-Toom B^T on integer codes is exact for m = 2, 4, 6; the factored form
-  // exists for F4 (F2's rows have two entries each: nothing to factor).
-  if (M == 4) return input_mode<M, kExact>(p, o.pdl, x, Vq, absmax, st);
-  return input_mode<M, kSparse>(p, o.pdl, x, Vq, absmax, st);
+  // Cook-Toom B^T on integer codes is exact for m = 2, 4, 6: factored forms throughout.
+  return input_mode<M, kExact>(p, o.pdl, x, Vq, absmax, st);
 }
 
 template <int M, int MODE, bool QM, int CPT>
@@ -344,7 +342,7 @@ int output_m(const Params& p, const LaunchOpt& o, float s_Y, const void* mbuf, c
   }
   // With Q_M on, the F4 output transform works on integers in [-128, 127]:
   // every intermediate is an integer below 2^24, so the factored form is exact.
-  if (M == 4 && qm) return output_mode<M, kExact, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st);
+  if (M != 6 && qm) return output_mode<M, kExact, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st);
   return qm ? output_mode<M, kSparse, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st)
             : output_mode<M, kSparse, false>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st);
 }

@@ -295,15 +295,14 @@ int WINO_CAT(launch_input_transform_tma_m, WINO_M)(const Params& p, const Launch
                                                     const CUtensorMap& mapV, int* status,
                                                     cudaStream_t st) {
   if (!o.std_mats) return input_tma_mode<WINO_M, kDense>(p, o.pdl, mapX, mapV, status, st);
-  if (WINO_M == 4) return input_tma_mode<WINO_M, kExact>(p, o.pdl, mapX, mapV, status, st);
-  return input_tma_mode<WINO_M, kSparse>(p, o.pdl, mapX, mapV, status, st);
+  return input_tma_mode<WINO_M, kExact>(p, o.pdl, mapX, mapV, status, st);
 }
 int WINO_CAT(launch_output_transform_tma_m, WINO_M)(const Params& p, const LaunchOpt& o,
                                                      const CUtensorMap& mapM,
                                                      const CUtensorMap& mapY, const float* bias,
                                                      float s_Y, int* status, cudaStream_t st) {
   if (!o.std_mats) return output_tma_mode<WINO_M, kDense>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
-  if (WINO_M == 4) return output_tma_mode<WINO_M, kExact>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
+  if (WINO_M != 6) return output_tma_mode<WINO_M, kExact>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
   return output_tma_mode<WINO_M, kSparse>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
 }
 
