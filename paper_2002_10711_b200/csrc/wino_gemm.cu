@@ -213,6 +213,10 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) tmem_alloc(tmem_slot, (uint32_t)a.tmem_cols);
+  if (warp == 0 && lane == 0) {   // descriptors do not depend on the previous kernel
+    tma_prefetch_map(&mapV);
+    tma_prefetch_map(&mapU);
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();

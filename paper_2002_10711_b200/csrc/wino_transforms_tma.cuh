@@ -67,6 +67,8 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   }
   __syncthreads();
   if (threadIdx.x == 0) {
+    tma_prefetch_map(&mapX);
+    tma_prefetch_map(&mapV);
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
     mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
     for (int i = 0; i < ntile; ++i) {
@@ -154,6 +156,8 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
   }
   __syncthreads();
   if (threadIdx.x == 0) {
+    tma_prefetch_map(&mapM);
+    tma_prefetch_map(&mapY);
     griddep_wait();
     mbar_expect_tx(bar, kInBytes);   // the full box counts, clipped rows included
     tma_load_3d(s_in, &mapM, bar, k0, tau0, 0);
