@@ -198,6 +198,24 @@ int wino_calibrate_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev,
                            const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
                            void* workspace_dev, uint32_t* absmax4_dev, void* stream);
 
+/* Direct int8 3x3 convolution (cross-correlation, zero padding 1, stride 1 or 2), the
+ * lossless candidate of the paper's search space (Section 4, "im2row") and the
+ * layer type of its strided convolutions, which have no Winograd form (Section
+ * 5.1).  acc = sum over the 3x3xC window of (x - z_x)(w - z_w) in int32 (padding
+ * is the real value zero); int8 output Q(fmaf((float)acc, (float)(s_x*s_w/s_Y),
+ * (float)(bias/s_Y)); 1), float output fmaf((float)acc, (float)(s_x*s_w), bias).
+ * x int8 [N][H][W][C], w int8 [K][3][3][C], y [N][Ho][Wo][K] with
+ * Ho = (H-1)/stride + 1; C and K multiples of 4; device pointers 16-byte aligned.
+ * Stateless: no plan, no workspace. */
+typedef struct {
+  int32_t N, C, H, W, K, stride;
+  wino_quant_t q_x, q_w, q_Y;
+  int32_t out_dtype;
+} wino_direct_desc_t;
+int wino_direct_conv_forward(const wino_direct_desc_t* desc, const int8_t* x_NHWC_dev,
+                             const int8_t* w_KRSC_dev, const float* bias_K_dev, void* y_dev,
+                             void* stream);
+
 /* Synchronizes `stream` and returns the plan's device status word: WINO_OK, or
  * WINO_ERR_TIMEOUT if a bounded wait inside a kernel expired (the kernel then
  * stopped early and its output is undefined), or WINO_ERR_CUDA. */

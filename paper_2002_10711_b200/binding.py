@@ -24,7 +24,7 @@ STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
 EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
-    "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages",
+    "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward", "wino_direct_conv_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages",
     "wino_launch_count", "wino_plan_set_stage_events", "wino_destroy", "wino_strerror",
 ]
 
@@ -41,6 +41,12 @@ class DescC(ct.Structure):
                 ("transforms_exact", ct.c_int32),
                 ("q_x", QuantC), ("q_w", QuantC), ("q_V", QuantC), ("q_U", QuantC),
                 ("q_M", QuantC), ("q_Y", QuantC), ("out_dtype", ct.c_int32)]
+
+
+class DirectDescC(ct.Structure):
+    _fields_ = [("N", ct.c_int32), ("C", ct.c_int32), ("H", ct.c_int32), ("W", ct.c_int32),
+                ("K", ct.c_int32), ("stride", ct.c_int32),
+                ("q_x", QuantC), ("q_w", QuantC), ("q_Y", QuantC), ("out_dtype", ct.c_int32)]
 
 
 class WinoError(RuntimeError):
@@ -69,6 +75,7 @@ def _load() -> ct.CDLL:
     lib.wino_conv_forward_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.wino_calibrate_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.wino_debug_run_stages.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
+    lib.wino_direct_conv_forward.argtypes = [ct.POINTER(DirectDescC), vp, vp, vp, vp, vp]
     lib.wino_last_status.argtypes = [vp, vp]
     lib.wino_debug_dump_stage.argtypes = [vp, i32, vp, sz]
     lib.wino_launch_count.argtypes = [vp]
@@ -114,6 +121,15 @@ def _stream_handle(stream) -> ct.c_void_p:
         import torch
         stream = torch.cuda.current_stream()
     return ct.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def direct_conv_forward(N, C, H, W, K, stride, q_x, q_w, q_Y, x_dev, w_dev, bias_dev, y_dev,
+                        out_dtype=0, stream=None) -> None:
+    """wino_direct_conv_forward: direct int8 3x3 convolution, stride 1 or 2."""
+    d = DirectDescC(N, C, H, W, K, stride, _quant(q_x), _quant(q_w), _quant(q_Y), out_dtype)
+    _check(_lib.wino_direct_conv_forward(ct.byref(d), _dptr(x_dev), _dptr(w_dev), _dptr(bias_dev),
+                                         _dptr(y_dev), _stream_handle(stream)),
+           "wino_direct_conv_forward")
 
 
 class Plan:

@@ -490,6 +490,25 @@ int wino_debug_run_stages(const wino_plan_t* pl, int stage_mask, const int8_t* x
   return forward_impl(pl, x, Uq, bias, y, ws, nullptr, (cudaStream_t)stream, stage_mask);
 }
 
+int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const int8_t* w,
+                             const float* bias, void* y, void* stream) {
+  if (d == nullptr || x == nullptr || w == nullptr || y == nullptr) return WINO_ERR_INVALID;
+  if (d->N < 1 || d->C < 1 || d->H < 1 || d->W < 1 || d->K < 1) return WINO_ERR_INVALID;
+  if (d->stride != 1 && d->stride != 2) return WINO_ERR_INVALID;
+  if (d->out_dtype != 0 && d->out_dtype != 1) return WINO_ERR_INVALID;
+  if (!quant_ok(d->q_x) || !quant_ok(d->q_w) || !quant_ok(d->q_Y)) return WINO_ERR_INVALID;
+  if (d->C % 4 != 0 || d->K % 4 != 0) return WINO_ERR_UNSUPPORTED;
+  if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias)))
+    return WINO_ERR_ALIGNMENT;
+  const double s_in = (double)d->q_x.scale * (double)d->q_w.scale;
+  return launch_direct_conv(d->N, d->C, d->H, d->W, d->K, d->stride, d->q_x.zero_point,
+                            d->q_w.zero_point, d->q_Y.zero_point,
+                            (float)(s_in / (double)d->q_Y.scale), (float)s_in, d->q_Y.scale,
+                            (float)(d->q_Y.qmin - d->q_Y.zero_point),
+                            (float)(d->q_Y.qmax - d->q_Y.zero_point), d->out_dtype, x, w, bias, y,
+                            (cudaStream_t)stream);
+}
+
 int wino_last_status(const wino_plan_t* pl, void* stream) {
   if (pl == nullptr) return WINO_ERR_INVALID;
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;

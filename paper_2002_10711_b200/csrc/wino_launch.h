@@ -51,6 +51,12 @@ int launch_fused_f2(const Params& p, const LaunchOpt& o, const CUtensorMap& mapU
                     const float* bias, void* y, float s_Y, int num_sms, int* status,
                     cudaStream_t st);
 
+// Direct int8 3x3 convolution (stride 1 or 2) on the ALUs.
+int launch_direct_conv(int N, int C, int H, int W, int K, int stride, int z_x, int z_w, int z_Y,
+                       float mult, float s_in, float s_Y, float lo_Y, float hi_Y, int out_dtype,
+                       const int8_t* x, const int8_t* w, const float* bias, void* y,
+                       cudaStream_t st);
+
 enum { kOutMq = 0, kOutI32 = 1 };
 constexpr int kBM = 128;      // tiles per GEMM block (MMA M)
 constexpr int kStageK = 128;  // channels (bytes) per shared-memory stage

@@ -1,0 +1,75 @@
+"""Direct int8 3x3 convolution on the GPU (stride 1 and 2) against the oracle's
+integer direct convolution and output quantizer: bit-exact int8 codes."""
+import numpy as np
+import pytest
+
+import oracle
+import wino_inputs as wi
+from oracle import Quant
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(N, C, H, W, K, stride, q_x, q_w, q_Y, x_q, w_q, bias, out_dtype=0):
+    import torch
+    from paper_2002_10711_b200 import binding
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    x = torch.from_numpy(x_q).cuda()
+    w = torch.from_numpy(w_q).cuda()
+    b = None if bias is None else torch.from_numpy(bias).cuda()
+    y = torch.empty((N, Ho, Wo, K), dtype=torch.float32 if out_dtype else torch.int8, device="cuda")
+    binding.direct_conv_forward(N, C, H, W, K, stride, q_x, q_w, q_Y, x, w, b, y, out_dtype=out_dtype)
+    torch.cuda.synchronize()
+    return y.cpu().numpy()
+
+
+@pytest.mark.parametrize("shape", [(2, 16, 9, 7, 8), (1, 64, 32, 32, 128), (3, 4, 1, 1, 4), (2, 128, 16, 16, 256),
+                                   (1, 20, 6, 11, 12)])
+@pytest.mark.parametrize("stride", [1, 2])
+@pytest.mark.parametrize("variant", ["plain", "relu_bias", "zero_points"])
+def test_direct_conv_matches_oracle(shape, stride, variant):
+    N, C, H, W, K = shape
+    x_q = wi.halfnormal_codes(5000 + C, 1, (N, H, W, C))
+    w_q, s_w = wi.gaussian_weight_codes(5000 + K, 2, (K, 3, 3, C), 0.05)
+    s_x = float(np.float32(1 / 32))
+    z_x = z_w = 0
+    bias = None
+    q_Y = Quant()
+    if variant == "relu_bias":
+        bias = wi.bias_values(5000, 3, K, 0.5)
+        q_Y = Quant(qmin=0)
+    if variant == "zero_points":
+        z_x, z_w = 4, -3
+        q_Y = Quant(zero_point=6)
+    acc = oracle.direct_conv_i32(x_q, w_q, z_x=z_x, z_w=z_w, stride=stride)
+    s_in = s_x * float(s_w)
+    q_Y.scale = float(np.float32(max(float(np.abs(acc).max()) * s_in, 1e-6) / 127.0))
+    want = oracle.requantize_acc(acc, s_in, q_Y, bias)
+    got = _run(N, C, H, W, K, stride, Quant(scale=s_x, zero_point=z_x), Quant(scale=float(s_w), zero_point=z_w),
+               q_Y, x_q, w_q, bias)
+    assert got.shape == want.shape and (got == want).all()
+    assert want.size < 100 or len(np.unique(want)) > 3
+
+
+def test_direct_conv_float_output():
+    N, C, H, W, K = 2, 32, 10, 9, 16
+    x_q = wi.halfnormal_codes(5100, 1, (N, H, W, C))
+    w_q, s_w = wi.gaussian_weight_codes(5100, 2, (K, 3, 3, C), 0.05)
+    bias = wi.bias_values(5100, 3, K, 0.5)
+    s_x = float(np.float32(1 / 32))
+    acc = oracle.direct_conv_i32(x_q, w_q, stride=2)
+    s_in = np.float32(s_x * float(s_w))
+    want = acc.astype(np.float32).astype(np.float64) * np.float64(s_in) + bias.astype(np.float64)
+    got = _run(N, C, H, W, K, 2, Quant(scale=s_x), Quant(scale=float(s_w)), Quant(), x_q, w_q, bias, out_dtype=1)
+    assert float(np.abs(got - want).max()) <= 1e-4 * float(np.abs(want).max())
+
+
+def test_direct_conv_argument_checks():
+    from paper_2002_10711_b200 import binding
+    q = Quant()
+    with pytest.raises(binding.WinoError) as e:
+        binding.direct_conv_forward(1, 16, 8, 8, 16, 3, q, q, q, 16, 16, None, 16, stream=0)
+    assert e.value.code == binding.ERR_INVALID
+    with pytest.raises(binding.WinoError) as e:
+        binding.direct_conv_forward(1, 6, 8, 8, 16, 1, q, q, q, 16, 16, None, 16, stream=0)
+    assert e.value.code == binding.ERR_UNSUPPORTED

@@ -1,7 +1,7 @@
 """cfg5: the sixteen 3x3 convolutions of a CIFAR-shaped ResNet-18 body chained
 conv -> ReLU -> conv in int8, tile size per stride-1 layer drawn from a seed
 (mimicking a searched per-layer assignment, paper Section 4).  Stride-2 layers
-are direct convolutions in the oracle.  Every Winograd layer's GPU output must
+are direct convolutions (oracle: integer definition; GPU: the library's direct kernel).  Every Winograd layer's GPU output must
 equal the oracle's byte for byte, both when fed the oracle's activations and
 when fed the GPU chain's own."""
 import numpy as np
@@ -35,7 +35,17 @@ def _run_chain(batch):
             real_max = float(np.abs(acc).max()) * s_x * float(s_w)
             q_Y = Quant(scale=float(np.float32(real_max / 127.0)), qmin=0)
             x_ref = oracle.requantize_acc(acc, s_x * float(s_w), q_Y)
-            x_gpu = x_ref.copy()      # not a Winograd layer: both chains take the oracle's result
+            # the GPU chain runs its strided layers with the library's direct convolution
+            import torch
+            from paper_2002_10711_b200 import binding
+            xd = torch.from_numpy(x_gpu).cuda()
+            wd = torch.from_numpy(w_q).cuda()
+            yd = torch.empty(x_ref.shape, dtype=torch.int8, device="cuda")
+            binding.direct_conv_forward(batch, spec["C"], spec["H"], spec["W"], spec["K"], 2,
+                                        Quant(scale=s_x), Quant(scale=float(s_w)), q_Y, xd, wd, None, yd)
+            torch.cuda.synchronize()
+            x_gpu = yd.cpu().numpy()
+            assert (x_gpu == x_ref).all(), f"layer {spec['index']} (direct, stride 2) differs"
             s_x = q_Y.scale
             continue
         m = spec["m"]
