@@ -23,14 +23,15 @@ int launch_output_transform(const Params& p, const LaunchOpt& o, float s_Y, cons
 int launch_gemm_dp4a(const Params& p, const LaunchOpt& o, const int8_t* Vq, const int8_t* Uq,
                      void* out, int out_mode, unsigned* absmaxM, cudaStream_t st);
 
-// TMA-staged transform kernels (input needs z_x == 0 and C % 64 == 0; output needs
-// Q_M on, int8 output and K % 64 == 0).  Channel chunk per block:
+// TMA-staged transform kernels (input needs z_x == 0 and C % 16 == 0; output needs
+// Q_M on, int8 output and K % 16 == 0).  Channel chunk per block:
 // (128 channels x 1 tile per block measured best on 256-channel layers: twice the
 // blocks of a 256-channel chunk, so the single wave balances over the SMs)
 inline int tma_chunk(int channels) {
-  return channels % 128 == 0 ? 128 : channels % 64 == 0 ? 64 : 0;
+  return channels % 128 == 0 ? 128 : channels % 64 == 0 ? 64 : channels % 32 == 0 ? 32
+       : channels % 16 == 0 ? 16 : 0;
 }
-inline int tma_group(int chunk) { return chunk == 128 ? 1 : 4; }
+inline int tma_group(int chunk) { return chunk == 128 ? 1 : chunk == 64 ? 4 : chunk == 32 ? 4 : 8; }
 int launch_input_transform_tma(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX,
                                const CUtensorMap& mapV, int* status, cudaStream_t st);
 int launch_output_transform_tma(const Params& p, const LaunchOpt& o, const CUtensorMap& mapM,

@@ -44,7 +44,8 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
                       const __grid_constant__ CUtensorMap mapV, int* __restrict__ status) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
-  constexpr uint32_t kUnitBytes = G * kTileBytes;
+  constexpr uint32_t kTileStride = (kTileBytes + 127u) & ~127u;   // TMA destinations stay 128-byte aligned
+  constexpr uint32_t kUnitBytes = G * kTileStride;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
   const uint32_t s_in = base;                 // [G][T2][CC]
@@ -76,7 +77,7 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
       const int tw = tau % p.TW;
       const int th = (tau / p.TW) % p.TH;
       const int n = tau / (p.TW * p.TH);
-      tma_load_4d(s_in + (uint32_t)i * kTileBytes, &mapX, bar, c0, tw * M - 1, th * M - 1, n);
+      tma_load_4d(s_in + (uint32_t)i * kTileStride, &mapX, bar, c0, tw * M - 1, th * M - 1, n);
     }
     // one thread polls (bounded); the others sleep in the barrier below
     if (!mbar_wait(bar, 0u, &abort_flag)) {
@@ -88,7 +89,7 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   if (*(volatile uint32_t*)&abort_flag != 0u) return;
   (void)mbar_try_wait(bar, 0u);   // every thread observes the completed phase itself
   if (g < ntile) {
-    const uint32_t rd = s_in + (uint32_t)g * kTileBytes + (uint32_t)(CPT * c4);
+    const uint32_t rd = s_in + (uint32_t)g * kTileStride + (uint32_t)(CPT * c4);
     uint32_t wd[T2];
 #pragma unroll
     for (int ab = 0; ab < T2; ++ab)
@@ -133,7 +134,8 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
                        float s_Y, int* __restrict__ status) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = KC / CPT;
   constexpr uint32_t kInBytes = T2 * G * KC;          // [T2][G][KC]
-  constexpr uint32_t kTileOut = M * M * KC;           // [M][M][KC] per tile
+  constexpr uint32_t kTileOutBytes = M * M * KC;      // [M][M][KC] per tile
+  constexpr uint32_t kTileOut = (kTileOutBytes + 127u) & ~127u;   // stride: TMA sources 128-byte aligned
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 127u) & ~127u;
   const uint32_t s_in = base;
@@ -220,8 +222,8 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
 }
 
 // ---------------------------------------------------------------------------
-// Launchers.  CC (or KC) is 128 when it divides the channel count (one tile per
-// block), else 64 (four tiles per block).
+// Launchers.  CC (or KC) is the largest of 128 / 64 / 32 / 16 that divides the
+// channel count; narrower chunks take several tiles per block.
 // ---------------------------------------------------------------------------
 namespace {
 
@@ -237,7 +239,7 @@ inline int tma_cpt(long tiles_times_channels) {
 template <int M, int MODE, int CC, int G, int CPT>
 int input_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
                      int* status, cudaStream_t st) {
-  constexpr size_t smem = 2 * (size_t)G * (M + 2) * (M + 2) * CC + 128 + 16;
+  constexpr size_t smem = 2 * (size_t)G * ((((M + 2) * (M + 2) * CC) + 127) / 128 * 128) + 128 + 16;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k_input_transform_tma<M, MODE, CC, G, CPT>,
@@ -255,18 +257,24 @@ int input_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapX, const CUt
   const int cc = tma_chunk(p.C);
   if (tma_cpt((long)p.T * p.C) == 4)
     return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 4>(p, pdl, mapX, mapV, status, st)
-                     : input_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapX, mapV, status, st);
+         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapX, mapV, status, st)
+         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 4>(p, pdl, mapX, mapV, status, st)
+                    : input_tma_launch<M, MODE, 16, 8, 4>(p, pdl, mapX, mapV, status, st);
   if (tma_cpt((long)p.T * p.C) == 1)
     return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 1>(p, pdl, mapX, mapV, status, st)
-                     : input_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapX, mapV, status, st);
+         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapX, mapV, status, st)
+         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 1>(p, pdl, mapX, mapV, status, st)
+                    : input_tma_launch<M, MODE, 16, 8, 1>(p, pdl, mapX, mapV, status, st);
   return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 2>(p, pdl, mapX, mapV, status, st)
-                     : input_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapX, mapV, status, st);
+         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapX, mapV, status, st)
+         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 2>(p, pdl, mapX, mapV, status, st)
+                    : input_tma_launch<M, MODE, 16, 8, 2>(p, pdl, mapX, mapV, status, st);
 }
 
 template <int M, int MODE, int KC, int G, int CPT>
 int output_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapM, const CUtensorMap& mapY,
                       const float* bias, float s_Y, int* status, cudaStream_t st) {
-  constexpr size_t smem = (size_t)G * ((M + 2) * (M + 2) + M * M) * KC + 128 + 16;
+  constexpr size_t smem = (size_t)G * ((M + 2) * (M + 2) * KC + ((M * M * KC + 127) / 128 * 128)) + 128 + 16;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(k_output_transform_tma<M, MODE, KC, G, CPT>,
@@ -284,12 +292,18 @@ int output_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapM, const CU
   const int kc = tma_chunk(p.K);
   if (tma_cpt((long)p.T * p.K) == 4)
     return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                     : output_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                    : output_tma_launch<M, MODE, 16, 8, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
   if (tma_cpt((long)p.T * p.K) == 1)
     return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                     : output_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                    : output_tma_launch<M, MODE, 16, 8, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st);
   return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                     : output_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
+                    : output_tma_launch<M, MODE, 16, 8, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st);
 }
 
 }  // namespace
