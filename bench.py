@@ -342,6 +342,22 @@ def run_ours(args, wl):
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
                         "traffic": NCU_TRAFFIC_CFG3.get(kernel_names[n]) if wl.name == "cfg3" else None,
                         "peak_note": f"of {peaks['source']}"}
+    # measured int8 tensor rate of this device: an MMA-only probe kernel (operands in
+    # shared memory, accumulators in tensor memory), timed with CUDA events
+    mma_probe = None
+    if rank == 0:
+        iters = 20000
+        plan.debug_mma_probe(200)
+        torch.cuda.synchronize()
+        p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        p0.record()
+        plan.debug_mma_probe(iters)
+        p1.record()
+        torch.cuda.synchronize()
+        sms = torch.cuda.get_device_properties(dev).multi_processor_count
+        mma_probe = sms * iters * 2.0 * 128 * 256 * 32 / (p0.elapsed_time(p1) * 1e-3) / 1e12
+        if roofline is not None and roofline["bound"] == "tensor":
+            roofline["frac_of_measured_int8_mma"] = roofline["achieved"] / mma_probe
     # whole-layer roofline of the path's definition: slower of MMA work at the int8
     # tensor peak and algorithmic bytes (x + y + U_q) at the HBM peak
     t_mma = wino_ops(wl, wl.N) / (2.0 * peaks["bf16_tflops"] * 1e12)
@@ -505,6 +521,7 @@ def run_ours(args, wl):
             "path": {1: "staged_tc", 2: "staged_dp4a", 3: "smallc", 4: "staged_tc_ptr", 5: "fused_f2"}[plan.path],
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "layer_roofline": layer_roof, "stages": stages,
+            "int8_mma_probe_TOPS": mma_probe,
             "weight_transform": {"us": wt_us, "GBps": wt_bytes / (wt_us * 1e-6) / 1e9,
                                  "algorithmic_bytes": wt_bytes},
             "overlapped_steps": overlapped,

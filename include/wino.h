@@ -237,6 +237,14 @@ int wino_debug_run_stages(const wino_plan_t* plan, int stage_mask, const int8_t*
                           const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
                           void* workspace_dev, void* stream);
 
+/* Tensor-pipe probe for the roofline of the Hadamard stage (the stage the paper calls
+ * the bulk of the computation, Section 1): launches, on every SM of the plan's device,
+ * `iters` back-to-back tcgen05 int8 MMAs of 128x256x32 on operands held in shared
+ * memory.  The work is iters * SMs * 2*128*256*32 operations; the caller times the
+ * launch (CUDA events) to get the sustained int8 tensor rate of the device.
+ * A bounded wait that expires is reported through wino_last_status. */
+int wino_debug_mma_probe(const wino_plan_t* plan, int iters, void* stream);
+
 /* Number of kernels launched by this plan since it was created. */
 long wino_launch_count(const wino_plan_t* plan);
 

@@ -24,7 +24,7 @@ STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
 EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
-    "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward", "wino_direct_conv_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages",
+    "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward", "wino_direct_conv_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages", "wino_debug_mma_probe",
     "wino_launch_count", "wino_plan_set_stage_events", "wino_destroy", "wino_strerror",
 ]
 
@@ -76,6 +76,7 @@ def _load() -> ct.CDLL:
     lib.wino_calibrate_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.wino_debug_run_stages.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.wino_direct_conv_forward.argtypes = [ct.POINTER(DirectDescC), vp, vp, vp, vp, vp]
+    lib.wino_debug_mma_probe.argtypes = [vp, i32, vp]
     lib.wino_last_status.argtypes = [vp, vp]
     lib.wino_debug_dump_stage.argtypes = [vp, i32, vp, sz]
     lib.wino_launch_count.argtypes = [vp]
@@ -214,6 +215,10 @@ class Plan:
         _check(_lib.wino_debug_run_stages(self._h, stage_mask, _dptr(x_dev), _dptr(Uq_dev),
                                           _dptr(bias_dev), _dptr(y_dev), _dptr(workspace_dev),
                                           _stream_handle(stream)), "wino_debug_run_stages")
+
+    def debug_mma_probe(self, iters: int, stream=None) -> None:
+        _check(_lib.wino_debug_mma_probe(self._h, iters, _stream_handle(stream)),
+               "wino_debug_mma_probe")
 
     def calibrate_forward(self, x_dev, Uq_dev, bias_dev, y_dev, workspace_dev, absmax4_dev,
                           stream=None) -> None:

@@ -509,6 +509,13 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
                             (cudaStream_t)stream);
 }
 
+int wino_debug_mma_probe(const wino_plan_t* pl, int iters, void* stream) {
+  if (pl == nullptr || iters < 1 || iters > (1 << 22)) return WINO_ERR_INVALID;
+  if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
+  pl->launches++;
+  return launch_mma_peak(iters, pl->num_sms, pl->status_dev, (cudaStream_t)stream);
+}
+
 int wino_last_status(const wino_plan_t* pl, void* stream) {
   if (pl == nullptr) return WINO_ERR_INVALID;
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;

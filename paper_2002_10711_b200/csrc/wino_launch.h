@@ -58,6 +58,9 @@ int launch_direct_conv(int N, int C, int H, int W, int K, int stride, int z_x, i
                        const int8_t* x, const int8_t* w, const float* bias, void* y,
                        cudaStream_t st);
 
+// Tensor-pipe probe: `iters` back-to-back 128x256x32 int8 MMAs on every SM.
+int launch_mma_peak(int iters, int num_sms, int* status, cudaStream_t st);
+
 enum { kOutMq = 0, kOutI32 = 1 };
 constexpr int kBM = 128;      // tiles per GEMM block (MMA M)
 constexpr int kStageK = 128;  // channels (bytes) per shared-memory stage

@@ -200,3 +200,15 @@ def test_gpu_calibration_matches_oracle_calibration():
         got = calibrate(make_plan, x_q, w_q, bias, L.q_x.scale, L.q_w.scale)
         want = (L.q_V.scale, L.q_U.scale, L.q_M.scale, L.q_Y.scale)
         assert tuple(np.float32(got)) == tuple(np.float32(want)), (name, got, want)
+
+
+def test_mma_probe_runs_and_reports_ok():
+    import torch
+    from paper_2002_10711_b200 import binding, cook_toom
+    BT, G, AT = cook_toom(4)
+    q = dict(scale=0.1)
+    plan = binding.Plan(2, 64, 8, 8, 64, 4, BT, G, AT, q, q, q, q, q, q)
+    plan.debug_mma_probe(500)
+    assert plan.last_status() == 0
+    with pytest.raises(binding.WinoError):
+        plan.debug_mma_probe(0)
