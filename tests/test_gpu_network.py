@@ -71,6 +71,12 @@ def test_resnet18_chain_small_batch():
     assert seen == {2, 4, 6}
 
 
+def test_resnet18_chain_full_batch():
+    # the configuration as stated: batch 256, all sixteen layers
+    seen = _run_chain(256)
+    assert seen == {2, 4, 6}
+
+
 @pytest.mark.parametrize("index", [0, 13])
 def test_resnet18_layer_full_batch(index):
     from gpu_helpers import gpu_run
