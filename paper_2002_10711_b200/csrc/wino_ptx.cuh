@@ -45,6 +45,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    // a spinning warp takes issue slots from the warps it waits for: back off
+    if (i > 8u) __nanosleep(i > 64u ? 128u : 32u);
     if ((i & 255u) == 0u) {
       if (*abort_flag != 0u) return false;
       if (clock64() - t0 > kWaitCycles) return false;
