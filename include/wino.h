@@ -49,8 +49,11 @@
  *
  * Devices and threads.  A plan belongs to the device that was current when
  * wino_plan ran (its status word lives there); use it with that device current.
- * A plan is not thread-safe: calls on one plan must not overlap in time on the
- * host.  Different plans may be used from different threads.
+ * Plans on several devices may coexist in one process.  A plan is not
+ * thread-safe: every call that launches work updates the plan (caches of
+ * tensor maps, launch counter), which is why those calls take a non-const
+ * plan; calls on one plan must not overlap in time on the host.  Different
+ * plans may be used from different threads.
  */
 #ifndef WINO_H_
 #define WINO_H_
@@ -139,12 +142,12 @@ int wino_plan_force_path(wino_plan_t* plan, int path);
  * out[0]=s_x/s_V, out[1]=s_w/s_U, out[2]=s_U*s_V/s_M, out[3]=s_acc/s_Y, out[4]=s_acc. */
 int wino_plan_multipliers(const wino_plan_t* plan, float out[5]);
 
-/* Weight transform U_q = Q(G g G^T) (paper: Eq. 1; done once per layer, "amortized
- * across inferences", Section 3.1).  w_KRSC_dev: int8 [K][3][3][C]; Uq_dev:
+/* Weight transform U_q = Q(G g G^T) (paper: Eq. 1; done once per layer, so its
+ * cost is spread over every later inference: Section 3.1).  w_KRSC_dev: int8 [K][3][3][C]; Uq_dev:
  * int8 [t*t][K][C]; both device pointers, 16-byte aligned.  absmax_dev
  * (nullable, device, one uint32 holding float bits, caller-zeroed) receives
  * max |U| before quantization, for calibration. */
-int wino_transform_weights(const wino_plan_t* plan, const int8_t* w_KRSC_dev, int8_t* Uq_dev,
+int wino_transform_weights(wino_plan_t* plan, const int8_t* w_KRSC_dev, int8_t* Uq_dev,
                            uint32_t* absmax_dev, void* stream);
 
 /* The forward pass (paper: Eq. 1 with the quantizers of Fig. 2): input
@@ -154,7 +157,7 @@ int wino_transform_weights(const wino_plan_t* plan, const int8_t* w_KRSC_dev, in
  * float [K] or NULL; y_NHWK_dev int8 or float [N][H][W][K] per out_dtype;
  * workspace_dev at least wino_workspace_bytes (may be NULL when that is 0).
  * All device pointers 16-byte aligned. */
-int wino_conv_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev, const int8_t* Uq_dev,
+int wino_conv_forward(wino_plan_t* plan, const int8_t* x_NHWC_dev, const int8_t* Uq_dev,
                       const float* bias_K_dev, void* y_NHWK_dev, void* workspace_dev,
                       void* stream);
 
@@ -173,9 +176,11 @@ int wino_conv_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev, const i
  * Same arguments, results and errors as wino_conv_forward, minus the workspace:
  * V_q and m_q live in a static device array of WINO_STATIC_SCRATCH_BYTES built
  * into the library (every GPU that loads the library holds those bytes until
- * the process exits).  A plan whose wino_workspace_bytes exceeds that size is
- * refused with WINO_ERR_WORKSPACE and nothing is launched.  The call makes no
- * cudaMalloc / cudaFree and uses no allocating library routine.
+ * the process exits).  A plan on a staged path whose wino_workspace_bytes
+ * exceeds that size is refused with WINO_ERR_WORKSPACE and nothing is launched;
+ * plans on a single-kernel path (WINO_PATH_SMALLC, WINO_PATH_FUSED_F2) need no
+ * scratch and are accepted at any size.  The call makes no cudaMalloc /
+ * cudaFree and uses no allocating library routine.
  *
  * First use on a device: the first call made with a given device current looks
  * up the array's device address (cudaGetSymbolAddress) and remembers it; make
@@ -185,7 +190,7 @@ int wino_conv_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev, const i
  * start at zero (each call overwrites every byte it later reads).  Two calls
  * whose kernels overlap on the GPU (different streams, no ordering between
  * them) race on the array and corrupt each other's result: order them. */
-int wino_conv_forward_static(const wino_plan_t* plan, const int8_t* x_NHWC_dev,
+int wino_conv_forward_static(wino_plan_t* plan, const int8_t* x_NHWC_dev,
                              const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
                              void* stream);
 
@@ -194,7 +199,7 @@ int wino_conv_forward_static(const wino_plan_t* plan, const int8_t* x_NHWC_dev,
  * in absmax4_dev[0..3] (device, caller-zeroed uint32[4]), the max-abs of
  * V (before Q_V), of M (as a float), of Y before the output scaling, and of
  * the float-mode output fmaf(Y, s_acc, bias).  y_NHWK_dev may be NULL. */
-int wino_calibrate_forward(const wino_plan_t* plan, const int8_t* x_NHWC_dev,
+int wino_calibrate_forward(wino_plan_t* plan, const int8_t* x_NHWC_dev,
                            const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
                            void* workspace_dev, uint32_t* absmax4_dev, void* stream);
 
@@ -218,22 +223,33 @@ int wino_direct_conv_forward(const wino_direct_desc_t* desc, const int8_t* x_NHW
 
 /* Synchronizes `stream` and returns the plan's device status word: WINO_OK, or
  * WINO_ERR_TIMEOUT if a bounded wait inside a kernel expired (the kernel then
- * stopped early and its output is undefined), or WINO_ERR_CUDA. */
-int wino_last_status(const wino_plan_t* plan, void* stream);
+ * stopped early and its output is undefined), or WINO_ERR_CUDA.  On the device
+ * the word is sticky (a later successful launch does not reset it); this call
+ * reads it and clears it, so the next call reports only what happened since. */
+int wino_last_status(wino_plan_t* plan, void* stream);
 
 /* Copies one intermediate of the most recent wino_conv_forward on this plan
  * (staged paths only) into dst_dev: V_q int8 [t*t][T][C], M int32 [t*t][T][K]
  * (recomputed from V_q and U_q with the plan's GEMM kernel), m_q int8
  * [t*t][T][K].  `bytes` must equal the stage size.  Asynchronous on the stream
  * of that forward call. */
-int wino_debug_dump_stage(const wino_plan_t* plan, int stage, void* dst_dev, size_t bytes);
+int wino_debug_dump_stage(wino_plan_t* plan, int stage, void* dst_dev, size_t bytes);
+
+/* The forward pass on a single-kernel path (WINO_PATH_SMALLC, WINO_PATH_FUSED_F2;
+ * WINO_ERR_UNSUPPORTED on the staged paths, which have wino_debug_dump_stage)
+ * that also writes the int32 Hadamard sums the kernel held in registers /
+ * tensor memory (paper: Eq. 1, the product inside the brackets, summed over
+ * channels) to M_dev, int32 [t*t][T][K]; `bytes` must equal that size. */
+int wino_debug_forward_accumulators(wino_plan_t* plan, const int8_t* x_NHWC_dev,
+                                    const int8_t* Uq_dev, const float* bias_K_dev,
+                                    void* y_NHWK_dev, int32_t* M_dev, size_t bytes, void* stream);
 
 /* Runs a subset of the three kernels of a staged path on the caller's buffers
  * (stages of the paper's Fig. 2): stage_mask bit 0 = input transform (x -> V_q in
  * the workspace), bit 1 = Hadamard GEMMs (V_q, U_q -> m_q in the workspace),
  * bit 2 = output transform (m_q -> y).  Stages left out read whatever an earlier
  * call left in the workspace.  For debugging and per-kernel timing. */
-int wino_debug_run_stages(const wino_plan_t* plan, int stage_mask, const int8_t* x_NHWC_dev,
+int wino_debug_run_stages(wino_plan_t* plan, int stage_mask, const int8_t* x_NHWC_dev,
                           const int8_t* Uq_dev, const float* bias_K_dev, void* y_NHWK_dev,
                           void* workspace_dev, void* stream);
 
@@ -243,17 +259,24 @@ int wino_debug_run_stages(const wino_plan_t* plan, int stage_mask, const int8_t*
  * memory.  The work is iters * SMs * 2*128*256*32 operations; the caller times the
  * launch (CUDA events) to get the sustained int8 tensor rate of the device.
  * A bounded wait that expires is reported through wino_last_status. */
-int wino_debug_mma_probe(const wino_plan_t* plan, int iters, void* stream);
+int wino_debug_mma_probe(wino_plan_t* plan, int iters, void* stream);
+
+/* Shows what every kernel of this library does when a barrier it waits for never
+ * completes (no counterpart in the paper).  Launches one small block that
+ * waits, for at most limit_cycles SM clocks (1 .. 1e8), on a barrier nothing
+ * arrives at, then records WINO_ERR_TIMEOUT in the plan's status word and exits
+ * normally; wino_last_status reports it and clears it, and the plan stays
+ * usable.  Production kernels use the same wait with a limit of about a second. */
+int wino_debug_wait_probe(wino_plan_t* plan, long long limit_cycles, void* stream);
+
+/* Host-side check of the library's once-per-device bookkeeping (kernel attributes
+ * are set once on every device a kernel runs on): returns 1 the first time it is
+ * called with a device index in [0, 64), 0 on later calls with the same index,
+ * WINO_ERR_INVALID outside the range.  Touches no GPU. */
+int wino_debug_once_per_device(int device);
 
 /* Number of kernels launched by this plan since it was created. */
 long wino_launch_count(const wino_plan_t* plan);
-
-/* Measurement hook for the staged paths (the stages are those of the paper's
- * Fig. 2): when set, every wino_conv_forward records the four caller-owned
- * cudaEvent_t handles on its stream: before the input transform, after it,
- * after the Hadamard-stage GEMMs, after the output transform.  NULL switches
- * the hook off.  The fused small-channel path records nothing. */
-int wino_plan_set_stage_events(wino_plan_t* plan, void* const events[4]);
 
 void wino_destroy(wino_plan_t* plan);
 const char* wino_strerror(int code);

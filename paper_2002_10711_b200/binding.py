@@ -24,8 +24,11 @@ STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
 EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
-    "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward", "wino_direct_conv_forward", "wino_last_status", "wino_debug_dump_stage", "wino_debug_run_stages", "wino_debug_mma_probe",
-    "wino_launch_count", "wino_plan_set_stage_events", "wino_destroy", "wino_strerror",
+    "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward",
+    "wino_direct_conv_forward", "wino_last_status", "wino_debug_dump_stage",
+    "wino_debug_forward_accumulators", "wino_debug_run_stages", "wino_debug_mma_probe",
+    "wino_debug_wait_probe", "wino_debug_once_per_device", "wino_launch_count", "wino_destroy",
+    "wino_strerror",
 ]
 
 
@@ -81,7 +84,9 @@ def _load() -> ct.CDLL:
     lib.wino_debug_dump_stage.argtypes = [vp, i32, vp, sz]
     lib.wino_launch_count.argtypes = [vp]
     lib.wino_launch_count.restype = ct.c_long
-    lib.wino_plan_set_stage_events.argtypes = [vp, vp]
+    lib.wino_debug_forward_accumulators.argtypes = [vp, vp, vp, vp, vp, vp, sz, vp]
+    lib.wino_debug_wait_probe.argtypes = [vp, ct.c_longlong, vp]
+    lib.wino_debug_once_per_device.argtypes = [i32]
     lib.wino_destroy.argtypes = [vp]
     lib.wino_destroy.restype = None
     lib.wino_strerror.argtypes = [i32]
@@ -122,6 +127,10 @@ def _stream_handle(stream) -> ct.c_void_p:
         import torch
         stream = torch.cuda.current_stream()
     return ct.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def debug_once_per_device(device: int) -> int:
+    return _lib.wino_debug_once_per_device(device)
 
 
 def direct_conv_forward(N, C, H, W, K, stride, q_x, q_w, q_Y, x_dev, w_dev, bias_dev, y_dev,
@@ -226,17 +235,19 @@ class Plan:
                                            _dptr(y_dev), _dptr(workspace_dev), _dptr(absmax4_dev),
                                            _stream_handle(stream)), "wino_calibrate_forward")
 
-    def set_stage_events(self, events) -> None:
-        """events: four cudaEvent_t handles (ints), or None to switch the hook off."""
-        if events is None:
-            _check(_lib.wino_plan_set_stage_events(self._h, None), "wino_plan_set_stage_events")
-            return
-        arr = (ct.c_void_p * 4)(*[ct.c_void_p(int(e)) for e in events])
-        self._stage_events = arr
-        _check(_lib.wino_plan_set_stage_events(self._h, ct.cast(arr, ct.c_void_p)),
-               "wino_plan_set_stage_events")
+    def debug_wait_probe(self, limit_cycles: int, stream=None) -> None:
+        _check(_lib.wino_debug_wait_probe(self._h, limit_cycles, _stream_handle(stream)),
+               "wino_debug_wait_probe")
+
+    def debug_forward_accumulators(self, x_dev, Uq_dev, bias_dev, y_dev, M_dev, nbytes: int,
+                                   stream=None) -> None:
+        _check(_lib.wino_debug_forward_accumulators(self._h, _dptr(x_dev), _dptr(Uq_dev),
+                                                    _dptr(bias_dev), _dptr(y_dev), _dptr(M_dev),
+                                                    nbytes, _stream_handle(stream)),
+               "wino_debug_forward_accumulators")
 
     def last_status(self, stream=None) -> int:
+        """Synchronizes the stream; returns the device status word and clears it."""
         return _lib.wino_last_status(self._h, _stream_handle(stream))
 
     def debug_dump_stage(self, stage: int, dst_dev, nbytes: int) -> None:

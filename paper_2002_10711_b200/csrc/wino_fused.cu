@@ -55,7 +55,7 @@ __device__ __forceinline__ void tmem_ld4(uint32_t taddr, uint32_t (&r)[4]) {
 __global__ void __launch_bounds__(kFusedThreads, 1)
 k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapU,
            const int8_t* __restrict__ x, const float* __restrict__ bias, void* __restrict__ y,
-           float s_Y, int n_mblk, int* __restrict__ status) {
+           float s_Y, int n_mblk, int* __restrict__ status, int* __restrict__ dbgM) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t sA = base;                         // 16 x kATile
@@ -240,6 +240,14 @@ k_fused_f2(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap
             for (int j = 0; j < 4; ++j)
               tmem_ld4(tlane + (uint32_t)((i * 4 + j) * 32 + sub * 8 + half * 4), acc[j]);
             tmem_ld_wait();
+            if (dbgM != nullptr && row_ok) {   // debugging aid: the int32 sums M[xi][tau][k]
+#pragma unroll
+              for (int j = 0; j < 4; ++j)
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                  if (kc + q < p.K)
+                    dbgM[((long)(i * 4 + j) * p.T + tau) * p.K + kc + q] = (int)acc[j][q];
+            }
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               float mrow[4];
@@ -317,20 +325,15 @@ bool fused_f2_supported(const Params& p, bool std_mats) {
 }
 
 int launch_fused_f2(const Params& p, const LaunchOpt& o, const CUtensorMap& mapU, const int8_t* x,
-                    const float* bias, void* y, float s_Y, int num_sms, int* status,
+                    const float* bias, void* y, float s_Y, int num_sms, int* status, int* dbgM,
                     cudaStream_t st) {
   const size_t smem = 1024 + 16 * (size_t)kATile + 16 * (size_t)kBTile + 256 + 128;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_fused_f2, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return -5;
-    attr_set = true;
-  }
+  static DeviceOnce once;
+  if (int rc = set_max_smem(once, o.device, k_fused_f2, smem)) return rc;
   const int n_mblk = (p.T + 127) / 128;
   const int grid = n_mblk < num_sms ? n_mblk : num_sms;
   return launch_kernel(k_fused_f2, dim3((unsigned)grid), dim3(kFusedThreads), smem, st, o.pdl, p,
-                       mapU, x, bias, y, s_Y, n_mblk, status);
+                       mapU, x, bias, y, s_Y, n_mblk, status, dbgM);
 }
 
 }  // namespace wino

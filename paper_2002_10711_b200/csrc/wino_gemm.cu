@@ -1,6 +1,6 @@
 // Hadamard stage of the Winograd-aware layer as t*t independent int8 GEMMs over
-// channels with int32 accumulation (paper: Sections 1 and 5.3, "element-wise
-// GEMM stage"):   M[xi][tau][k] = sum_c V_q[xi][tau][c] * U_q[xi][k][c]
+// channels with int32 accumulation (paper: Sections 1 and 5.3, where the
+// position-wise products are carried out as GEMMs):   M[xi][tau][k] = sum_c V_q[xi][tau][c] * U_q[xi][k][c]
 // followed by the quantizer of the Hadamard output (paper: Fig. 2).
 //
 //   k_gemm_tc   : persistent, warp-specialised tcgen05 kernel.  int8 operands are
@@ -331,13 +331,8 @@ TcGeom tc_geometry(const Params& p, int num_sms) {
 int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,
                    const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
                    int* status, cudaStream_t st) {
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024) !=
-        cudaSuccess)
-      return -5;
-    attr_set = true;
-  }
+  static DeviceOnce once;
+  if (int rc = set_max_smem(once, o.device, k_gemm_tc, 227 * 1024)) return rc;
   GemmTcArgs a;
   a.BN = g.BN; a.stages = g.stages; a.tmem_cols = g.tmem_cols; a.acc_stride = g.tmem_cols / 2;
   a.out_mode = out_mode;

@@ -47,20 +47,19 @@ struct wino_plan {
   int path;
   int* status_dev;      // device status word (may be null when no GPU is present)
   int num_sms;
+  int device;           // the device that was current when the plan was made
   bool pdl;             // programmatic dependent launch between the stages
   // memo of the last encoded tensor maps
-  mutable const void* map_vq_ptr;
-  mutable const void* map_uq_ptr;
-  mutable CUtensorMap mapV, mapU;
+  const void* map_vq_ptr;
+  const void* map_uq_ptr;
+  CUtensorMap mapV, mapU;
   // maps of the TMA-staged transform kernels, keyed by buffer address
-  mutable MapCache cache_x, cache_vst, cache_mld, cache_y, cache_uf;
+  MapCache cache_x, cache_vst, cache_mld, cache_y, cache_uf;
   // last forward call, for wino_debug_dump_stage
-  mutable const int8_t* last_uq;
-  mutable void* last_ws;
-  mutable cudaStream_t last_stream;
-  mutable long launches;
-  cudaEvent_t stage_ev[4];  // caller-owned; recorded around the three staged kernels when set
-  bool stage_ev_on;
+  const int8_t* last_uq;
+  void* last_ws;
+  cudaStream_t last_stream;
+  long launches;
 };
 
 // Scratch of wino_conv_forward_static: V_q and m_q of one layer call.  A plain
@@ -94,18 +93,18 @@ int static_scratch_address(void** out) {
   return WINO_OK;
 }
 
+EncodeTiledFn lookup_encode_fn() {
+  void* ptr = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) ==
+          cudaSuccess &&
+      q == cudaDriverEntryPointSuccess)
+    return reinterpret_cast<EncodeTiledFn>(ptr);
+  cudaGetLastError();
+  return nullptr;
+}
 EncodeTiledFn get_encode_fn() {
-  static EncodeTiledFn fn = nullptr;
-  static bool tried = false;
-  if (!tried) {
-    tried = true;
-    void* ptr = nullptr;
-    cudaDriverEntryPointQueryResult q;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) ==
-            cudaSuccess &&
-        q == cudaDriverEntryPointSuccess)
-      fn = reinterpret_cast<EncodeTiledFn>(ptr);
-  }
+  static const EncodeTiledFn fn = lookup_encode_fn();   // initialised once, thread-safe
   return fn;
 }
 
@@ -149,6 +148,7 @@ LaunchOpt opt_of(const wino_plan_t* pl, bool pdl) {
   LaunchOpt o;
   o.std_mats = pl->std_mats;
   o.pdl = pdl;
+  o.device = pl->device;
   return o;
 }
 
@@ -179,7 +179,7 @@ int encode_map(CUtensorMap* map, const void* base, uint64_t inner, uint64_t rows
 }
 
 // Tensor maps of the TMA-staged transform kernels (no swizzle).
-const CUtensorMap* map_x(const wino_plan_t* pl, const void* x) {
+const CUtensorMap* map_x(wino_plan_t* pl, const void* x) {
   if (const CUtensorMap* m = pl->cache_x.find(x)) return m;
   const Params& p = pl->p;
   const uint64_t dims[4] = {(uint64_t)p.C, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.N};
@@ -191,7 +191,7 @@ const CUtensorMap* map_x(const wino_plan_t* pl, const void* x) {
   }
   return m;
 }
-const CUtensorMap* map_y(const wino_plan_t* pl, const void* y) {
+const CUtensorMap* map_y(wino_plan_t* pl, const void* y) {
   if (const CUtensorMap* m = pl->cache_y.find(y)) return m;
   const Params& p = pl->p;
   const uint64_t dims[4] = {(uint64_t)p.K, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.N};
@@ -204,7 +204,7 @@ const CUtensorMap* map_y(const wino_plan_t* pl, const void* y) {
   return m;
 }
 // V_q (store side) and m_q (load side): [t*t][T][channels], box {chunk, G, t*t}
-const CUtensorMap* map_stage(const wino_plan_t* pl, MapCache& cache, const void* buf, int channels) {
+const CUtensorMap* map_stage(wino_plan_t* pl, MapCache& cache, const void* buf, int channels) {
   if (const CUtensorMap* m = cache.find(buf)) return m;
   const Params& p = pl->p;
   const int chunk = tma_chunk(channels);
@@ -219,7 +219,7 @@ const CUtensorMap* map_stage(const wino_plan_t* pl, MapCache& cache, const void*
 }
 
 // U_q for the fused F2 kernel: [16][K][C], box {64, 64, 1}, 64-byte swizzle
-const CUtensorMap* map_u_fused(const wino_plan_t* pl, const void* Uq) {
+const CUtensorMap* map_u_fused(wino_plan_t* pl, const void* Uq) {
   if (const CUtensorMap* m = pl->cache_uf.find(Uq)) return m;
   const Params& p = pl->p;
   const uint64_t dims[3] = {(uint64_t)p.C, (uint64_t)p.K, 16};
@@ -232,7 +232,7 @@ const CUtensorMap* map_u_fused(const wino_plan_t* pl, const void* Uq) {
   return m;
 }
 
-int launch_gemm(const wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void* out, int out_mode,
+int launch_gemm(wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void* out, int out_mode,
                 unsigned* absmaxM, bool pdl, cudaStream_t st) {
   const Params& p = pl->p;
   const int t2 = p.t * p.t;
@@ -254,37 +254,34 @@ int launch_gemm(const wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void*
                         pl->status_dev, st);
 }
 
-// stage_mask: bit 0 input transform, bit 1 Hadamard GEMMs, bit 2 output transform
-int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias, void* y,
-                 void* ws, unsigned* absmax4, cudaStream_t st, int stage_mask = 7) {
+// stage_mask: bit 0 input transform, bit 1 Hadamard GEMMs, bit 2 output transform.
+// dbgM (single-kernel paths only): receives the int32 Hadamard sums M[xi][tau][k].
+int forward_impl(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias, void* y,
+                 void* ws, unsigned* absmax4, cudaStream_t st, int stage_mask = 7,
+                 int* dbgM = nullptr) {
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
   const bool calib = absmax4 != nullptr;
   const bool pdl = pl->pdl && !calib;
   if (pl->path == WINO_PATH_SMALLC && !calib) {
     pl->launches++;
-    return launch_smallc(pl->p, opt_of(pl, pdl), x, Uq, bias, y, pl->s_Y, st);
+    return launch_smallc(pl->p, opt_of(pl, pdl), x, Uq, bias, y, pl->s_Y, dbgM, st);
   }
   if (pl->path == WINO_PATH_FUSED_F2 && !calib && stage_mask == 7) {
     const CUtensorMap* mu = map_u_fused(pl, Uq);
     if (mu == nullptr) return WINO_ERR_CUDA;
     pl->launches++;
     return launch_fused_f2(pl->p, opt_of(pl, pdl), *mu, x, bias, y, pl->s_Y, pl->num_sms,
-                           pl->status_dev, st);
+                           pl->status_dev, dbgM, st);
   }
   if (ws == nullptr) return WINO_ERR_WORKSPACE;
   if (!aligned16(ws)) return WINO_ERR_ALIGNMENT;
   int8_t* Vq = reinterpret_cast<int8_t*>(ws);
   void* mbuf = reinterpret_cast<uint8_t*>(ws) + round_up(vq_bytes(pl), 1024);
-  // calibration on a small-channel plan uses the dp4a kernel for the middle stage
-  wino_plan_t tmp_holder;
-  const wino_plan_t* run = pl;
-  if (pl->path == WINO_PATH_SMALLC || pl->path == WINO_PATH_FUSED_F2) {
-    tmp_holder = *pl;
-    tmp_holder.path = pl->path == WINO_PATH_SMALLC ? WINO_PATH_STAGED_DP4A : WINO_PATH_STAGED_TC_PTR;
-    run = &tmp_holder;
-  }
-  const bool ev = pl->stage_ev_on;
-  if (ev) cudaEventRecord(pl->stage_ev[0], st);
+  // calibration on a single-kernel plan runs the staged kernels (dp4a or tcgen05 middle stage)
+  const int saved_path = pl->path;
+  int gemm_path = pl->path;
+  if (pl->path == WINO_PATH_SMALLC) gemm_path = WINO_PATH_STAGED_DP4A;
+  if (pl->path == WINO_PATH_FUSED_F2) gemm_path = WINO_PATH_STAGED_TC_PTR;
   const bool tma_ok = pl->path == WINO_PATH_STAGED_TC && !calib;
   int rc = WINO_OK;
   if (!(stage_mask & 1)) {
@@ -292,40 +289,41 @@ int forward_impl(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const
     const CUtensorMap* mx = map_x(pl, x);
     const CUtensorMap* mv = map_stage(pl, pl->cache_vst, Vq, pl->p.C);
     if (mx == nullptr || mv == nullptr) return WINO_ERR_CUDA;
-    rc = launch_input_transform_tma(pl->p, opt_of(pl, pdl && !ev), *mx, *mv, pl->status_dev, st);
+    rc = launch_input_transform_tma(pl->p, opt_of(pl, pdl), *mx, *mv, pl->status_dev, st);
   } else {
-    rc = launch_input_transform(pl->p, opt_of(pl, pdl && !ev), x, Vq, calib ? absmax4 + 0 : nullptr,
-                                st);
+    rc = launch_input_transform(pl->p, opt_of(pl, pdl), x, Vq, calib ? absmax4 + 0 : nullptr, st);
   }
   if (rc != WINO_OK) return rc;
-  if (ev) cudaEventRecord(pl->stage_ev[1], st);
   if (stage_mask & 2) {
-    rc = launch_gemm(run, Vq, Uq, mbuf, pl->p.qM_enabled ? kOutMq : kOutI32,
-                     calib ? absmax4 + 1 : nullptr, pdl && !ev, st);
-    if (run != pl) {
-      pl->launches++;
-    }
+    pl->path = gemm_path;
+    rc = launch_gemm(pl, Vq, Uq, mbuf, pl->p.qM_enabled ? kOutMq : kOutI32,
+                     calib ? absmax4 + 1 : nullptr, pdl, st);
+    pl->path = saved_path;
   }
   if (rc != WINO_OK) return rc;
-  if (ev) cudaEventRecord(pl->stage_ev[2], st);
   if (!(stage_mask & 4)) {
   } else if (pl->launches++, tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
     const CUtensorMap* mm = map_stage(pl, pl->cache_mld, mbuf, pl->p.K);
     const CUtensorMap* my = map_y(pl, y);
     if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
-    rc = launch_output_transform_tma(pl->p, opt_of(pl, pdl && !ev), *mm, *my, bias, pl->s_Y,
+    rc = launch_output_transform_tma(pl->p, opt_of(pl, pdl), *mm, *my, bias, pl->s_Y,
                                      pl->status_dev, st);
   } else {
-    rc = launch_output_transform(pl->p, opt_of(pl, pdl && !ev), pl->s_Y, mbuf, bias, y,
+    rc = launch_output_transform(pl->p, opt_of(pl, pdl), pl->s_Y, mbuf, bias, y,
                                  calib ? absmax4 + 2 : nullptr, st);
   }
   if (rc != WINO_OK) return rc;
-  if (ev) cudaEventRecord(pl->stage_ev[3], st);
   pl->last_uq = Uq;
   pl->last_ws = ws;
   pl->last_stream = st;
   return WINO_OK;
 }
+
+bool path_uses_scratch(const wino_plan_t* pl) {
+  return pl->path != WINO_PATH_SMALLC && pl->path != WINO_PATH_FUSED_F2;
+}
+
+DeviceOnce g_once_selftest;
 
 }  // namespace
 
@@ -400,8 +398,9 @@ int wino_plan(const wino_desc_t* desc, wino_plan_t** out) {
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) == cudaSuccess && ndev > 0) {
     int dev = 0, sms = 0;
-    if (cudaGetDevice(&dev) == cudaSuccess &&
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess && sms > 0)
+    if (cudaGetDevice(&dev) == cudaSuccess) pl->device = dev;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, pl->device) == cudaSuccess &&
+        sms > 0)
       pl->num_sms = sms;
     if (cudaMalloc(&pl->status_dev, 256) == cudaSuccess) {
       cudaMemset(pl->status_dev, 0, 256);
@@ -442,7 +441,7 @@ int wino_plan_multipliers(const wino_plan_t* pl, float out[5]) {
   return WINO_OK;
 }
 
-int wino_transform_weights(const wino_plan_t* pl, const int8_t* w, int8_t* Uq, uint32_t* absmax,
+int wino_transform_weights(wino_plan_t* pl, const int8_t* w, int8_t* Uq, uint32_t* absmax,
                            void* stream) {
   if (pl == nullptr || w == nullptr || Uq == nullptr) return WINO_ERR_INVALID;
   if (!aligned16(w) || !aligned16(Uq)) return WINO_ERR_ALIGNMENT;
@@ -451,7 +450,7 @@ int wino_transform_weights(const wino_plan_t* pl, const int8_t* w, int8_t* Uq, u
   return launch_weight_transform(pl->p, w, Uq, absmax, (cudaStream_t)stream);
 }
 
-int wino_conv_forward(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias,
+int wino_conv_forward(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias,
                       void* y, void* ws, void* stream) {
   if (pl == nullptr || x == nullptr || Uq == nullptr || y == nullptr) return WINO_ERR_INVALID;
   if (!aligned16(x) || !aligned16(Uq) || !aligned16(y) || (bias && !aligned16(bias)))
@@ -459,19 +458,21 @@ int wino_conv_forward(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq, 
   return forward_impl(pl, x, Uq, bias, y, ws, nullptr, (cudaStream_t)stream);
 }
 
-int wino_conv_forward_static(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq,
+int wino_conv_forward_static(wino_plan_t* pl, const int8_t* x, const int8_t* Uq,
                              const float* bias, void* y, void* stream) {
   if (pl == nullptr || x == nullptr || Uq == nullptr || y == nullptr) return WINO_ERR_INVALID;
   if (!aligned16(x) || !aligned16(Uq) || !aligned16(y) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
-  if (wino_workspace_bytes(pl) > (size_t)WINO_STATIC_SCRATCH_BYTES) return WINO_ERR_WORKSPACE;
   void* scratch = nullptr;
-  const int rc = static_scratch_address(&scratch);
-  if (rc != WINO_OK) return rc;
+  if (path_uses_scratch(pl)) {   // the single-kernel paths keep V_q and m_q on the SM
+    if (wino_workspace_bytes(pl) > (size_t)WINO_STATIC_SCRATCH_BYTES) return WINO_ERR_WORKSPACE;
+    const int rc = static_scratch_address(&scratch);
+    if (rc != WINO_OK) return rc;
+  }
   return forward_impl(pl, x, Uq, bias, y, scratch, nullptr, (cudaStream_t)stream);
 }
 
-int wino_calibrate_forward(const wino_plan_t* pl, const int8_t* x, const int8_t* Uq,
+int wino_calibrate_forward(wino_plan_t* pl, const int8_t* x, const int8_t* Uq,
                            const float* bias, void* y, void* ws, uint32_t* absmax4, void* stream) {
   if (pl == nullptr || x == nullptr || Uq == nullptr || absmax4 == nullptr) return WINO_ERR_INVALID;
   if (!aligned16(x) || !aligned16(Uq) || (y && !aligned16(y)) || (bias && !aligned16(bias)))
@@ -479,7 +480,7 @@ int wino_calibrate_forward(const wino_plan_t* pl, const int8_t* x, const int8_t*
   return forward_impl(pl, x, Uq, bias, y, ws, absmax4, (cudaStream_t)stream);
 }
 
-int wino_debug_run_stages(const wino_plan_t* pl, int stage_mask, const int8_t* x, const int8_t* Uq,
+int wino_debug_run_stages(wino_plan_t* pl, int stage_mask, const int8_t* x, const int8_t* Uq,
                           const float* bias, void* y, void* ws, void* stream) {
   if (pl == nullptr || x == nullptr || Uq == nullptr || y == nullptr) return WINO_ERR_INVALID;
   if (stage_mask < 1 || stage_mask > 7) return WINO_ERR_INVALID;
@@ -509,24 +510,53 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
                             (cudaStream_t)stream);
 }
 
-int wino_debug_mma_probe(const wino_plan_t* pl, int iters, void* stream) {
+int wino_debug_mma_probe(wino_plan_t* pl, int iters, void* stream) {
   if (pl == nullptr || iters < 1 || iters > (1 << 22)) return WINO_ERR_INVALID;
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
   pl->launches++;
-  return launch_mma_peak(iters, pl->num_sms, pl->status_dev, (cudaStream_t)stream);
+  return launch_mma_peak(iters, pl->num_sms, pl->device, pl->status_dev, (cudaStream_t)stream);
 }
 
-int wino_last_status(const wino_plan_t* pl, void* stream) {
+int wino_debug_wait_probe(wino_plan_t* pl, long long limit_cycles, void* stream) {
+  if (pl == nullptr || limit_cycles < 1 || limit_cycles > 100000000ll) return WINO_ERR_INVALID;
+  if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
+  pl->launches++;
+  return launch_wait_probe(limit_cycles, pl->status_dev, (cudaStream_t)stream);
+}
+
+int wino_debug_forward_accumulators(wino_plan_t* pl, const int8_t* x, const int8_t* Uq,
+                                    const float* bias, void* y, int32_t* M_dev, size_t bytes,
+                                    void* stream) {
+  if (pl == nullptr || x == nullptr || Uq == nullptr || y == nullptr || M_dev == nullptr)
+    return WINO_ERR_INVALID;
+  if (path_uses_scratch(pl)) return WINO_ERR_UNSUPPORTED;   // staged paths: wino_debug_dump_stage
+  if (bytes != m_elems(pl) * 4) return WINO_ERR_INVALID;
+  if (!aligned16(x) || !aligned16(Uq) || !aligned16(y) || !aligned16(M_dev) ||
+      (bias && !aligned16(bias)))
+    return WINO_ERR_ALIGNMENT;
+  return forward_impl(pl, x, Uq, bias, y, nullptr, nullptr, (cudaStream_t)stream, 7, M_dev);
+}
+
+int wino_debug_once_per_device(int device) {
+  if (device < 0 || device >= DeviceOnce::kMaxDevices) return WINO_ERR_INVALID;
+  int ran = 0;
+  g_once_selftest.run(device, [&]() -> int { ran = 1; return 0; });
+  return ran;
+}
+
+int wino_last_status(wino_plan_t* pl, void* stream) {
   if (pl == nullptr) return WINO_ERR_INVALID;
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
   if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return WINO_ERR_CUDA;
   int v = 0;
   if (cudaMemcpy(&v, pl->status_dev, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
     return WINO_ERR_CUDA;
+  // read and clear: the word is sticky on the device, the next read starts afresh
+  if (v != 0 && cudaMemset(pl->status_dev, 0, sizeof(int)) != cudaSuccess) return WINO_ERR_CUDA;
   return v;
 }
 
-int wino_debug_dump_stage(const wino_plan_t* pl, int stage, void* dst, size_t bytes) {
+int wino_debug_dump_stage(wino_plan_t* pl, int stage, void* dst, size_t bytes) {
   if (pl == nullptr || dst == nullptr) return WINO_ERR_INVALID;
   if (pl->last_ws == nullptr) return WINO_ERR_UNSUPPORTED;
   if (!aligned16(dst)) return WINO_ERR_ALIGNMENT;
@@ -545,30 +575,18 @@ int wino_debug_dump_stage(const wino_plan_t* pl, int stage, void* dst, size_t by
   }
   if (stage == WINO_STAGE_M_I32) {
     if (bytes != m_elems(pl) * 4) return WINO_ERR_INVALID;
-    wino_plan_t tmp = *pl;
-    if (tmp.path == WINO_PATH_SMALLC) tmp.path = WINO_PATH_STAGED_DP4A;
-    int rc = launch_gemm(&tmp, reinterpret_cast<const int8_t*>(ws), pl->last_uq, dst, kOutI32,
-                         nullptr, false, st);
-    pl->launches++;
-    pl->map_vq_ptr = tmp.map_vq_ptr; pl->map_uq_ptr = tmp.map_uq_ptr;
-    pl->mapV = tmp.mapV; pl->mapU = tmp.mapU;
+    const int saved_path = pl->path;
+    if (pl->path == WINO_PATH_SMALLC) pl->path = WINO_PATH_STAGED_DP4A;
+    if (pl->path == WINO_PATH_FUSED_F2) pl->path = WINO_PATH_STAGED_TC_PTR;
+    const int rc = launch_gemm(pl, reinterpret_cast<const int8_t*>(ws), pl->last_uq, dst, kOutI32,
+                               nullptr, false, st);
+    pl->path = saved_path;
     return rc;
   }
   return WINO_ERR_INVALID;
 }
 
 long wino_launch_count(const wino_plan_t* pl) { return pl ? pl->launches : 0; }
-
-int wino_plan_set_stage_events(wino_plan_t* pl, void* const events[4]) {
-  if (pl == nullptr) return WINO_ERR_INVALID;
-  if (events == nullptr) { pl->stage_ev_on = false; return WINO_OK; }
-  for (int i = 0; i < 4; ++i) {
-    if (events[i] == nullptr) return WINO_ERR_INVALID;
-    pl->stage_ev[i] = (cudaEvent_t)events[i];
-  }
-  pl->stage_ev_on = true;
-  return WINO_OK;
-}
 
 void wino_destroy(wino_plan_t* pl) {
   if (pl == nullptr) return;

@@ -2,6 +2,8 @@
 // translation units.  Every function enqueues work on `st` and returns 0 or a
 // negative WINO_ERR_* code; none allocates or synchronizes.
 #pragma once
+#include <mutex>
+
 #include <cuda.h>
 #include <cuda_runtime.h>
 #include "wino_common.cuh"
@@ -12,7 +14,40 @@ namespace wino {
 struct LaunchOpt {
   bool std_mats = false;      // B^T and A^T are the built-in Cook-Toom matrices
   bool pdl = false;           // programmatic dependent launch on the stream
+  int device = 0;             // the plan's device (current when the launcher runs)
 };
+
+// "Done once per device" bookkeeping.  cudaFuncSetAttribute applies to the device
+// that is current when it is called, so the opt-in to more than 48 KB of dynamic
+// shared memory has to be repeated on every device a kernel is launched on.
+// run(dev, fn) calls fn() the first time it sees `dev` (and again if fn failed)
+// under a lock, so concurrent first launches from several host threads are safe.
+// Device indices beyond the table always run fn.
+class DeviceOnce {
+ public:
+  static constexpr int kMaxDevices = 64;
+  template <typename Fn>
+  int run(int dev, Fn fn) {
+    if (dev < 0 || dev >= kMaxDevices) return fn();
+    std::lock_guard<std::mutex> lock(mu_);
+    if (done_[dev]) return 0;
+    const int rc = fn();
+    if (rc == 0) done_[dev] = true;
+    return rc;
+  }
+ private:
+  std::mutex mu_;
+  bool done_[kMaxDevices] = {};
+};
+
+// Opt a kernel in to `smem` bytes of dynamic shared memory on device `dev`.
+template <typename Kern>
+int set_max_smem(DeviceOnce& once, int dev, Kern kernel, size_t smem) {
+  return once.run(dev, [&]() -> int {
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) ==
+                   cudaSuccess ? 0 : -5;
+  });
+}
 
 int launch_weight_transform(const Params& p, const int8_t* w, int8_t* Uq, unsigned* absmax,
                             cudaStream_t st);
@@ -44,12 +79,12 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
                    const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
                    int* status, cudaStream_t st);
 int launch_smallc(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
-                  const float* bias, void* y, float s_Y, cudaStream_t st);
+                  const float* bias, void* y, float s_Y, int* dbgM, cudaStream_t st);
 
 // Fully fused F2 kernel for narrow layers (C in {32, 64}, K <= 64, Cook-Toom matrices).
 bool fused_f2_supported(const Params& p, bool std_mats);
 int launch_fused_f2(const Params& p, const LaunchOpt& o, const CUtensorMap& mapU, const int8_t* x,
-                    const float* bias, void* y, float s_Y, int num_sms, int* status,
+                    const float* bias, void* y, float s_Y, int num_sms, int* status, int* dbgM,
                     cudaStream_t st);
 
 // Direct int8 3x3 convolution (stride 1 or 2) on the ALUs.
@@ -59,7 +94,11 @@ int launch_direct_conv(int N, int C, int H, int W, int K, int stride, int z_x, i
                        cudaStream_t st);
 
 // Tensor-pipe probe: `iters` back-to-back 128x256x32 int8 MMAs on every SM.
-int launch_mma_peak(int iters, int num_sms, int* status, cudaStream_t st);
+int launch_mma_peak(int iters, int num_sms, int device, int* status, cudaStream_t st);
+
+// Bounded-wait probe: one block waits, with the given cycle limit, on a barrier
+// that nothing arrives at, records WINO_ERR_TIMEOUT in *status and exits normally.
+int launch_wait_probe(long long limit_cycles, int* status, cudaStream_t st);
 
 enum { kOutMq = 0, kOutI32 = 1 };
 constexpr int kBM = 128;      // tiles per GEMM block (MMA M)

@@ -1,3 +1,5 @@
+// Debug probes.
+//
 // Tensor-pipe probe: how many int8 multiply-accumulates per second the tcgen05
 // kind::i8 MMA sustains on this device when nothing else is in the way.  One CTA
 // per SM, operands resident in shared memory (zeros), one thread issues a long
@@ -50,16 +52,40 @@ k_mma_peak(int iters, int* __restrict__ status) {
   }
 }
 
-int launch_mma_peak(int iters, int num_sms, int* status, cudaStream_t st) {
+int launch_mma_peak(int iters, int num_sms, int device, int* status, cudaStream_t st) {
   const size_t smem = 1024 + (128 + 256) * 128 + 64;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_mma_peak, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return -5;
-    attr_set = true;
-  }
+  static DeviceOnce once;
+  if (int rc = set_max_smem(once, device, k_mma_peak, smem)) return rc;
   return launch_kernel(k_mma_peak, dim3((unsigned)num_sms), dim3(128), smem, st, false, iters, status);
+}
+
+// Bounded-wait probe: what a production kernel does when a barrier it waits for
+// never completes, without making a production kernel fail.  One block, nothing
+// in flight, no tensor memory held: thread 0 waits (same mbar_wait as every
+// kernel, with the caller's cycle limit) on a barrier nobody arrives at, records
+// WINO_ERR_TIMEOUT and the block leaves by its normal exit.
+__global__ void __launch_bounds__(32)
+k_wait_probe(long long limit_cycles, int* __restrict__ status) {
+  __shared__ __align__(8) unsigned long long bar_storage;
+  __shared__ uint32_t abort_flag;
+  const uint32_t bar = smem_u32(&bar_storage);
+  if (threadIdx.x == 0) {
+    mbar_init(bar, 1);
+    abort_flag = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncwarp();
+  if (threadIdx.x == 0) {
+    if (!mbar_wait(bar, 0u, &abort_flag, limit_cycles)) {
+      abort_flag = 1u;
+      atomicExch(status, -6);   // WINO_ERR_TIMEOUT
+    }
+  }
+  __syncwarp();
+}
+
+int launch_wait_probe(long long limit_cycles, int* status, cudaStream_t st) {
+  return launch_kernel(k_wait_probe, dim3(1), dim3(32), 0, st, false, limit_cycles, status);
 }
 
 }  // namespace wino

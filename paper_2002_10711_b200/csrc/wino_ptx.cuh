@@ -40,7 +40,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // raises the abort flag and unwinds; the host reads WINO_ERR_TIMEOUT.
 constexpr long long kWaitCycles = 2000000000ll;
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
-                                          volatile uint32_t* abort_flag) {
+                                          volatile uint32_t* abort_flag,
+                                          long long limit_cycles = kWaitCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
@@ -49,7 +50,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
     if (i > 8u) __nanosleep(i > 64u ? 128u : 32u);
     if ((i & 255u) == 0u) {
       if (*abort_flag != 0u) return false;
-      if (clock64() - t0 > kWaitCycles) return false;
+      if (clock64() - t0 > limit_cycles) return false;
     }
   }
 }

@@ -21,7 +21,7 @@ template <int M, bool STD, int LPT>
 __global__ void __launch_bounds__(128)
 k_smallc(const __grid_constant__ Params p, const int8_t* __restrict__ x,
          const int8_t* __restrict__ Uq, const float* __restrict__ bias, void* __restrict__ y,
-         float s_Y) {
+         float s_Y, int* __restrict__ dbgM) {
   constexpr int T_ = M + 2, T2 = T_ * T_;
   constexpr int TPW = 32 / LPT;                   // tiles per warp
   constexpr int MODE = STD ? kSparse : kDense;
@@ -96,6 +96,8 @@ k_smallc(const __grid_constant__ Params p, const int8_t* __restrict__ x,
         const int vv = (int)__shfl_sync(0xffffffffu, w4, tbase + 4 * L);
         macc = __dp4a(vv, (int)su[(xi * L4 + L) * LPT], macc);
       }
+      // debugging aid: the int32 Hadamard sum itself, M[xi][tau][k]
+      if (dbgM != nullptr && k_ok && t_ok) dbgM[((long)xi * p.T + tau) * K + l] = macc;
       float mval = __int2float_rn(macc);
       if (p.qM_enabled) mval = magic_to_float(quant_magic(mval, p.mult_M, p.lo_M, p.hi_M));
       mf[xi] = mval;
@@ -131,43 +133,39 @@ k_smallc(const __grid_constant__ Params p, const int8_t* __restrict__ x,
 namespace {
 
 template <int M, bool STD, int LPT>
-int smallc_launch(const Params& p, bool pdl, const int8_t* x, const int8_t* Uq, const float* bias,
-                  void* y, float s_Y, cudaStream_t st) {
+int smallc_launch(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq, const float* bias,
+                  void* y, float s_Y, int* dbgM, cudaStream_t st) {
   constexpr int T2 = (M + 2) * (M + 2);
   const size_t smem = (size_t)T2 * (LPT / 4) * LPT * 4;
-  static bool attr_set = false;   // one flag per instantiation
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_smallc<M, STD, LPT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)smem) != cudaSuccess) return -5;
-    attr_set = true;
-  }
+  static DeviceOnce once;   // one per instantiation
+  if (int rc = set_max_smem(once, o.device, k_smallc<M, STD, LPT>, smem)) return rc;
   const int groups = (p.T + (32 / LPT) - 1) / (32 / LPT);
   int blocks = (groups + 3) / 4;
   if (blocks > 148 * 8) blocks = 148 * 8;
-  return launch_kernel(k_smallc<M, STD, LPT>, dim3((unsigned)blocks), dim3(128), smem, st, pdl, p, x,
-                       Uq, bias, y, s_Y);
+  return launch_kernel(k_smallc<M, STD, LPT>, dim3((unsigned)blocks), dim3(128), smem, st, o.pdl, p, x,
+                       Uq, bias, y, s_Y, dbgM);
 }
 template <int M, bool STD>
-int smallc_lpt(const Params& p, bool pdl, const int8_t* x, const int8_t* Uq, const float* bias,
-               void* y, float s_Y, cudaStream_t st) {
+int smallc_lpt(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq, const float* bias,
+               void* y, float s_Y, int* dbgM, cudaStream_t st) {
   const int wide = p.C > p.K ? p.C : p.K;
-  return wide <= 8  ? smallc_launch<M, STD, 8>(p, pdl, x, Uq, bias, y, s_Y, st)
-       : wide <= 16 ? smallc_launch<M, STD, 16>(p, pdl, x, Uq, bias, y, s_Y, st)
-                    : smallc_launch<M, STD, 32>(p, pdl, x, Uq, bias, y, s_Y, st);
+  return wide <= 8  ? smallc_launch<M, STD, 8>(p, o, x, Uq, bias, y, s_Y, dbgM, st)
+       : wide <= 16 ? smallc_launch<M, STD, 16>(p, o, x, Uq, bias, y, s_Y, dbgM, st)
+                    : smallc_launch<M, STD, 32>(p, o, x, Uq, bias, y, s_Y, dbgM, st);
 }
 template <int M>
 int smallc_m(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
-             const float* bias, void* y, float s_Y, cudaStream_t st) {
-  return o.std_mats ? smallc_lpt<M, true>(p, o.pdl, x, Uq, bias, y, s_Y, st)
-                    : smallc_lpt<M, false>(p, o.pdl, x, Uq, bias, y, s_Y, st);
+             const float* bias, void* y, float s_Y, int* dbgM, cudaStream_t st) {
+  return o.std_mats ? smallc_lpt<M, true>(p, o, x, Uq, bias, y, s_Y, dbgM, st)
+                    : smallc_lpt<M, false>(p, o, x, Uq, bias, y, s_Y, dbgM, st);
 }
 }  // namespace
 
 int launch_smallc(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
-                  const float* bias, void* y, float s_Y, cudaStream_t st) {
-  return p.m == 2 ? smallc_m<2>(p, o, x, Uq, bias, y, s_Y, st)
-       : p.m == 4 ? smallc_m<4>(p, o, x, Uq, bias, y, s_Y, st)
-                  : smallc_m<6>(p, o, x, Uq, bias, y, s_Y, st);
+                  const float* bias, void* y, float s_Y, int* dbgM, cudaStream_t st) {
+  return p.m == 2 ? smallc_m<2>(p, o, x, Uq, bias, y, s_Y, dbgM, st)
+       : p.m == 4 ? smallc_m<4>(p, o, x, Uq, bias, y, s_Y, dbgM, st)
+                  : smallc_m<6>(p, o, x, Uq, bias, y, s_Y, dbgM, st);
 }
 
 }  // namespace wino

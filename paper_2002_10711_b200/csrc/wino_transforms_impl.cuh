@@ -260,8 +260,6 @@ namespace {
 // Channels per thread: the widest element that still gives every SM several
 // warps of work (148 SMs x 1024 threads as the target).
 int pick_cpt(long items_times_channels) {
-  static const int forced = [] { const char* e = getenv("WINO_CPT"); return e ? atoi(e) : 0; }();
-  if (forced == 1 || forced == 2 || forced == 4) return forced;
   const long target = 148l * 1024;
   if (items_times_channels / 4 >= target) return 4;
   if (items_times_channels / 2 >= target) return 2;

@@ -336,92 +336,80 @@ namespace {
 // most resident warps) and no byte-insert step; it is used unless the grid is so
 // large that four channels per thread still fill every SM many warps deep.
 inline int tma_cpt(long tiles_times_channels) {
-  static const int forced = [] { const char* e = getenv("WINO_TMA_CPT"); return e ? atoi(e) : 0; }();
-  if (forced == 1 || forced == 2 || forced == 4) return forced;
   return tiles_times_channels / (4 * 32) >= 148l * 64 ? 4 : 1;
 }
 
 template <int M, int MODE, int CC, int G, int CPT, int UPB>
-int input_tma_launch_u(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
+int input_tma_launch_u(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX, const CUtensorMap& mapV,
                        int* status, cudaStream_t st) {
   constexpr size_t smem =
       2 * (size_t)UPB * G * ((((M + 2) * (M + 2) * CC) + 127) / 128 * 128) + 128 + 16 * UPB;
   auto kernel = UPB == 1 ? k_input_transform_tma<M, MODE, CC, G, CPT>
                          : k_input_transform_tma_multi<M, MODE, CC, G, CPT, UPB>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
-        cudaSuccess)
-      return -5;
-    attr_set = true;
-  }
+  static DeviceOnce once;   // one per instantiation
+  if (int rc = set_max_smem(once, o.device, kernel, smem)) return rc;
   const int units = ((p.T + G - 1) / G) * (p.C / CC);
   return launch_kernel(kernel, dim3((unsigned)((units + UPB - 1) / UPB)), dim3((CC / CPT) * G), smem,
-                       st, pdl, p, mapX, mapV, status);
+                       st, o.pdl, p, mapX, mapV, status);
 }
 template <int M, int MODE, int CC, int G, int CPT>
-int input_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
+int input_tma_launch(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX, const CUtensorMap& mapV,
                      int* status, cudaStream_t st) {
   // two units per block once the grid is several waves deep (measured: 8 % faster at four
   // times the cfg3 batch, 15 % slower at the cfg3 batch itself)
   const long threads = (long)((p.T + G - 1) / G) * (p.C / CC) * ((CC / CPT) * G);
   if (threads >= 3l * 148 * 2048)
-    return input_tma_launch_u<M, MODE, CC, G, CPT, 2>(p, pdl, mapX, mapV, status, st);
-  return input_tma_launch_u<M, MODE, CC, G, CPT, 1>(p, pdl, mapX, mapV, status, st);
+    return input_tma_launch_u<M, MODE, CC, G, CPT, 2>(p, o, mapX, mapV, status, st);
+  return input_tma_launch_u<M, MODE, CC, G, CPT, 1>(p, o, mapX, mapV, status, st);
 }
 template <int M, int MODE>
-int input_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapX, const CUtensorMap& mapV,
+int input_tma_mode(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX, const CUtensorMap& mapV,
                    int* status, cudaStream_t st) {
   const int cc = tma_chunk(p.C);
   if (tma_cpt((long)p.T * p.C) == 4)
-    return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 4>(p, pdl, mapX, mapV, status, st)
-         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapX, mapV, status, st)
-         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 4>(p, pdl, mapX, mapV, status, st)
-                    : input_tma_launch<M, MODE, 16, 8, 4>(p, pdl, mapX, mapV, status, st);
+    return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 4>(p, o, mapX, mapV, status, st)
+         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 4>(p, o, mapX, mapV, status, st)
+         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 4>(p, o, mapX, mapV, status, st)
+                    : input_tma_launch<M, MODE, 16, 8, 4>(p, o, mapX, mapV, status, st);
   if (tma_cpt((long)p.T * p.C) == 1)
-    return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 1>(p, pdl, mapX, mapV, status, st)
-         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapX, mapV, status, st)
-         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 1>(p, pdl, mapX, mapV, status, st)
-                    : input_tma_launch<M, MODE, 16, 8, 1>(p, pdl, mapX, mapV, status, st);
-  return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 2>(p, pdl, mapX, mapV, status, st)
-         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapX, mapV, status, st)
-         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 2>(p, pdl, mapX, mapV, status, st)
-                    : input_tma_launch<M, MODE, 16, 8, 2>(p, pdl, mapX, mapV, status, st);
+    return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 1>(p, o, mapX, mapV, status, st)
+         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 1>(p, o, mapX, mapV, status, st)
+         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 1>(p, o, mapX, mapV, status, st)
+                    : input_tma_launch<M, MODE, 16, 8, 1>(p, o, mapX, mapV, status, st);
+  return cc == 128 ? input_tma_launch<M, MODE, 128, 1, 2>(p, o, mapX, mapV, status, st)
+         : cc == 64 ? input_tma_launch<M, MODE, 64, 4, 2>(p, o, mapX, mapV, status, st)
+         : cc == 32 ? input_tma_launch<M, MODE, 32, 4, 2>(p, o, mapX, mapV, status, st)
+                    : input_tma_launch<M, MODE, 16, 8, 2>(p, o, mapX, mapV, status, st);
 }
 
 template <int M, int MODE, int KC, int G, int CPT>
-int output_tma_launch(const Params& p, bool pdl, const CUtensorMap& mapM, const CUtensorMap& mapY,
+int output_tma_launch(const Params& p, const LaunchOpt& o, const CUtensorMap& mapM, const CUtensorMap& mapY,
                       const float* bias, float s_Y, int* status, cudaStream_t st) {
   constexpr size_t smem = (size_t)G * ((M + 2) * (M + 2) * KC + ((M * M * KC + 127) / 128 * 128)) + 128 + 16;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(k_output_transform_tma<M, MODE, KC, G, CPT>,
-                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
-      return -5;
-    attr_set = true;
-  }
+  static DeviceOnce once;   // one per instantiation
+  if (int rc = set_max_smem(once, o.device, k_output_transform_tma<M, MODE, KC, G, CPT>, smem)) return rc;
   const int units = ((p.T + G - 1) / G) * (p.K / KC);
   return launch_kernel(k_output_transform_tma<M, MODE, KC, G, CPT>, dim3((unsigned)units),
-                       dim3((KC / CPT) * G), smem, st, pdl, p, mapM, mapY, bias, s_Y, status);
+                       dim3((KC / CPT) * G), smem, st, o.pdl, p, mapM, mapY, bias, s_Y, status);
 }
 template <int M, int MODE>
-int output_tma_mode(const Params& p, bool pdl, const CUtensorMap& mapM, const CUtensorMap& mapY,
+int output_tma_mode(const Params& p, const LaunchOpt& o, const CUtensorMap& mapM, const CUtensorMap& mapY,
                     const float* bias, float s_Y, int* status, cudaStream_t st) {
   const int kc = tma_chunk(p.K);
   if (tma_cpt((long)p.T * p.K) == 4)
-    return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                    : output_tma_launch<M, MODE, 16, 8, 4>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+    return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 4>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 4>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 4>(p, o, mapM, mapY, bias, s_Y, status, st)
+                    : output_tma_launch<M, MODE, 16, 8, 4>(p, o, mapM, mapY, bias, s_Y, status, st);
   if (tma_cpt((long)p.T * p.K) == 1)
-    return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                    : output_tma_launch<M, MODE, 16, 8, 1>(p, pdl, mapM, mapY, bias, s_Y, status, st);
-  return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st)
-                    : output_tma_launch<M, MODE, 16, 8, 2>(p, pdl, mapM, mapY, bias, s_Y, status, st);
+    return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 1>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 1>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 1>(p, o, mapM, mapY, bias, s_Y, status, st)
+                    : output_tma_launch<M, MODE, 16, 8, 1>(p, o, mapM, mapY, bias, s_Y, status, st);
+  return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 2>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 2>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 2>(p, o, mapM, mapY, bias, s_Y, status, st)
+                    : output_tma_launch<M, MODE, 16, 8, 2>(p, o, mapM, mapY, bias, s_Y, status, st);
 }
 
 }  // namespace
@@ -430,16 +418,16 @@ int WINO_CAT(launch_input_transform_tma_m, WINO_M)(const Params& p, const Launch
                                                     const CUtensorMap& mapX,
                                                     const CUtensorMap& mapV, int* status,
                                                     cudaStream_t st) {
-  if (!o.std_mats) return input_tma_mode<WINO_M, kDense>(p, o.pdl, mapX, mapV, status, st);
-  return input_tma_mode<WINO_M, kExact>(p, o.pdl, mapX, mapV, status, st);
+  if (!o.std_mats) return input_tma_mode<WINO_M, kDense>(p, o, mapX, mapV, status, st);
+  return input_tma_mode<WINO_M, kExact>(p, o, mapX, mapV, status, st);
 }
 int WINO_CAT(launch_output_transform_tma_m, WINO_M)(const Params& p, const LaunchOpt& o,
                                                      const CUtensorMap& mapM,
                                                      const CUtensorMap& mapY, const float* bias,
                                                      float s_Y, int* status, cudaStream_t st) {
-  if (!o.std_mats) return output_tma_mode<WINO_M, kDense>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
-  if (WINO_M != 6) return output_tma_mode<WINO_M, kExact>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
-  return output_tma_mode<WINO_M, kSparse>(p, o.pdl, mapM, mapY, bias, s_Y, status, st);
+  if (!o.std_mats) return output_tma_mode<WINO_M, kDense>(p, o, mapM, mapY, bias, s_Y, status, st);
+  if (WINO_M != 6) return output_tma_mode<WINO_M, kExact>(p, o, mapM, mapY, bias, s_Y, status, st);
+  return output_tma_mode<WINO_M, kSparse>(p, o, mapM, mapY, bias, s_Y, status, st);
 }
 
 }  // namespace wino

@@ -19,6 +19,14 @@ def gpu_run(L, x_q, w_q, bias, path=binding.PATH_AUTO, dumps=False):
     assert st == 0, binding.strerror(st)
     out = {"y": y.cpu().numpy(), "U_q": conv.Uq.cpu().numpy().reshape(L.t * L.t, L.K, L.C),
            "path": plan.path, "launches": plan.launch_count}
+    if plan.path in (binding.PATH_SMALLC, binding.PATH_FUSED_F2):
+        # single-kernel paths: a second pass that also writes the int32 Hadamard sums
+        M = torch.full((L.t * L.t, plan.T, L.K), -1, dtype=torch.int32, device="cuda")
+        y2 = conv.empty_output()
+        plan.debug_forward_accumulators(x, conv.Uq, conv.bias, y2, M, M.numel() * 4)
+        assert plan.last_status() == 0
+        assert torch.equal(y2, y)
+        out["M"] = M.cpu().numpy()
     if dumps:
         out["V_q"] = conv.dump(binding.STAGE_VQ).cpu().numpy()
         out["M"] = conv.dump(binding.STAGE_M_I32).cpu().numpy()

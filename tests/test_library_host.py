@@ -110,3 +110,15 @@ def test_null_and_alignment_checks_without_gpu():
     assert lib.wino_transform_weights(p._h, 16, 33, None, None) == binding.ERR_ALIGNMENT
     assert lib.wino_debug_dump_stage(p._h, 0, 16, 10) == binding.ERR_UNSUPPORTED  # no forward yet
     assert binding.strerror(binding.ERR_TIMEOUT).startswith("bounded")
+
+
+def test_once_per_device_bookkeeping():
+    # kernel attributes are set once on every device a kernel runs on: the table is keyed
+    # by device index, so a second device gets its own first time
+    assert binding.debug_once_per_device(3) == 1
+    assert binding.debug_once_per_device(3) == 0
+    assert binding.debug_once_per_device(4) == 1
+    assert binding.debug_once_per_device(3) == 0
+    assert binding.debug_once_per_device(63) == 1
+    assert binding.debug_once_per_device(64) == binding.ERR_INVALID
+    assert binding.debug_once_per_device(-1) == binding.ERR_INVALID
