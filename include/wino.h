@@ -82,7 +82,12 @@ enum {
   WINO_PATH_STAGED_DP4A = 2, /* transform kernels + integer-dot-product GEMMs on the ALUs */
   WINO_PATH_SMALLC = 3,      /* one fused warp-shuffle kernel, C <= 32 and K <= 32 (never chosen automatically) */
   WINO_PATH_STAGED_TC_PTR = 4, /* as 1, but always the pointer-based transform kernels */
-  WINO_PATH_FUSED_F2 = 5     /* one fused tcgen05 kernel: m = 2, Cook-Toom matrices, C in {32, 64}, K <= 64 */
+  WINO_PATH_FUSED_F2 = 5,    /* one fused tcgen05 kernel: m = 2, Cook-Toom matrices, C in {32, 64}, K <= 64 */
+  WINO_PATH_STAGED_TC_MMA = 6, /* as 1, with the transforms themselves on the tensor cores where that is
+                                 exact: Cook-Toom F2 / F4, channel counts multiples of 128 */
+  WINO_PATH_FUSED_LAYER = 7   /* the whole layer in one persistent launch (tensor-core transforms and
+                                 GEMMs; V_q and m_q pass through the workspace in L2): Cook-Toom F2 / F4,
+                                 C and K multiples of 128, input zero point 0, Q_M on, int8 output */
 };
 
 /* Stages that wino_debug_dump_stage can copy out (staged paths only). */

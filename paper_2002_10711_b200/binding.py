@@ -18,6 +18,8 @@ WINO_OK = 0
 ERR_INVALID, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -1, -2, -3, -4, -5, -6
 PATH_AUTO, PATH_STAGED_TC, PATH_STAGED_DP4A, PATH_SMALLC, PATH_STAGED_TC_PTR = 0, 1, 2, 3, 4
 PATH_FUSED_F2 = 5
+PATH_STAGED_TC_MMA = 6
+PATH_FUSED_LAYER = 7
 STAGE_VQ, STAGE_M_I32, STAGE_MQ = 0, 1, 2
 STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
 

@@ -277,9 +277,9 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     }
   } else {
     // epilogue warps.  small: |M| <= 127^2 * C < 2^22; full: every 32-column chunk
-    // lies inside K.
+    // of every column block lies inside K (the last block is not ragged).
     const bool small = p.C <= 260;
-    const bool full = (p.K % 32) == 0 && (a.BN % 32) == 0;
+    const bool full = (p.K % a.BN) == 0 && (a.BN % 32) == 0;
     if (absmaxM != nullptr)
       epilogue_loop<false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
                                         abort_p, warp, lane);

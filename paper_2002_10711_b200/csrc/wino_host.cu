@@ -46,6 +46,11 @@ struct wino_plan {
   bool std_mats;        // BT and AT equal the built-in Cook-Toom matrices bit for bit
   int path;
   int* status_dev;      // device status word (may be null when no GPU is present)
+  void* kron_dev;       // Kronecker tables of the tensor-core transforms (same allocation)
+  unsigned* counters_dev;  // progress counters of the single-launch layer kernel (same allocation)
+  CUtensorMap fmapV, fmapU;   // GEMM operand maps of the single-launch kernel
+  const void* fmap_vq_ptr;
+  const void* fmap_uq_ptr;
   int num_sms;
   int device;           // the device that was current when the plan was made
   bool pdl;             // programmatic dependent launch between the stages
@@ -54,7 +59,7 @@ struct wino_plan {
   const void* map_uq_ptr;
   CUtensorMap mapV, mapU;
   // maps of the TMA-staged transform kernels, keyed by buffer address
-  MapCache cache_x, cache_vst, cache_mld, cache_y, cache_uf;
+  MapCache cache_x, cache_vst, cache_mld, cache_y, cache_uf, cache_x_sw, cache_m_sw;
   // last forward call, for wino_debug_dump_stage
   const int8_t* last_uq;
   void* last_ws;
@@ -132,10 +137,14 @@ bool path_supported(const wino_plan_t* pl, int path) {
   const int C = pl->d.C, K = pl->d.K;
   switch (path) {
     case WINO_PATH_STAGED_TC:
+    case WINO_PATH_STAGED_TC_MMA:
     case WINO_PATH_STAGED_TC_PTR: return C % 16 == 0 && K % 16 == 0;
     case WINO_PATH_STAGED_DP4A: return C % 4 == 0 && K % 4 == 0;
     case WINO_PATH_SMALLC: return C % 4 == 0 && K % 4 == 0 && C <= 32 && K <= 32;
     case WINO_PATH_FUSED_F2: return fused_f2_supported(pl->p, pl->std_mats);
+    case WINO_PATH_FUSED_LAYER:
+      return layer_fused_supported(pl->p, pl->std_mats) &&
+             layer_fused_geometry(pl->p, pl->num_sms).stages >= 2;
     default: return false;
   }
 }
@@ -218,6 +227,33 @@ const CUtensorMap* map_stage(wino_plan_t* pl, MapCache& cache, const void* buf, 
   return m;
 }
 
+// Swizzled maps of the tensor-core transform kernels: x as [N][H][W][C] with box
+// {128, t, t, 1}; m_q as [t*t][T][K] with box {128, 1, t*t}.
+const CUtensorMap* map_x_sw(wino_plan_t* pl, const void* x) {
+  if (const CUtensorMap* m = pl->cache_x_sw.find(x)) return m;
+  const Params& p = pl->p;
+  const uint64_t dims[4] = {(uint64_t)p.C, (uint64_t)p.W, (uint64_t)p.H, (uint64_t)p.N};
+  const uint32_t box[4] = {128, (uint32_t)p.t, (uint32_t)p.t, 1};
+  CUtensorMap* m = pl->cache_x_sw.slot(x);
+  if (encode_tiled(m, x, 4, dims, box, CU_TENSOR_MAP_SWIZZLE_128B) != WINO_OK) {
+    pl->cache_x_sw.key[(pl->cache_x_sw.next + MapCache::kN - 1) % MapCache::kN] = nullptr;
+    return nullptr;
+  }
+  return m;
+}
+const CUtensorMap* map_m_sw(wino_plan_t* pl, const void* mbuf) {
+  if (const CUtensorMap* m = pl->cache_m_sw.find(mbuf)) return m;
+  const Params& p = pl->p;
+  const uint64_t dims[3] = {(uint64_t)p.K, (uint64_t)p.T, (uint64_t)(p.t * p.t)};
+  const uint32_t box[3] = {128, 1, (uint32_t)(p.t * p.t)};
+  CUtensorMap* m = pl->cache_m_sw.slot(mbuf);
+  if (encode_tiled(m, mbuf, 3, dims, box, CU_TENSOR_MAP_SWIZZLE_128B) != WINO_OK) {
+    pl->cache_m_sw.key[(pl->cache_m_sw.next + MapCache::kN - 1) % MapCache::kN] = nullptr;
+    return nullptr;
+  }
+  return m;
+}
+
 // U_q for the fused F2 kernel: [16][K][C], box {64, 64, 1}, 64-byte swizzle
 const CUtensorMap* map_u_fused(wino_plan_t* pl, const void* Uq) {
   if (const CUtensorMap* m = pl->cache_uf.find(Uq)) return m;
@@ -277,15 +313,57 @@ int forward_impl(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float
   if (!aligned16(ws)) return WINO_ERR_ALIGNMENT;
   int8_t* Vq = reinterpret_cast<int8_t*>(ws);
   void* mbuf = reinterpret_cast<uint8_t*>(ws) + round_up(vq_bytes(pl), 1024);
+  if (pl->path == WINO_PATH_FUSED_LAYER && !calib && stage_mask == 7) {
+    const Params& p = pl->p;
+    const FusedGeom g = layer_fused_geometry(p, pl->num_sms);
+    const int t2 = p.t * p.t;
+    if (pl->fmap_vq_ptr != Vq) {
+      int rc = encode_map(&pl->fmapV, Vq, (uint64_t)p.C, (uint64_t)p.T, (uint64_t)t2, kBM);
+      if (rc != WINO_OK) return rc;
+      pl->fmap_vq_ptr = Vq;
+    }
+    if (pl->fmap_uq_ptr != Uq) {
+      int rc = encode_map(&pl->fmapU, Uq, (uint64_t)p.C, (uint64_t)p.K, (uint64_t)t2, (uint32_t)g.BN);
+      if (rc != WINO_OK) return rc;
+      pl->fmap_uq_ptr = Uq;
+    }
+    FusedMaps m;
+    m.x = map_x_sw(pl, x);
+    m.v_store = map_stage(pl, pl->cache_vst, Vq, p.C);
+    m.v_load = &pl->fmapV;
+    m.u = &pl->fmapU;
+    m.m_load = map_m_sw(pl, mbuf);
+    m.y = map_y(pl, y);
+    if (m.x == nullptr || m.v_store == nullptr || m.m_load == nullptr || m.y == nullptr)
+      return WINO_ERR_CUDA;
+    pl->launches++;
+    const int rc = launch_layer_fused(p, opt_of(pl, pdl), g, m, pl->kron_dev, pl->counters_dev,
+                                      reinterpret_cast<int8_t*>(mbuf), bias, pl->s_Y,
+                                      pl->status_dev, st);
+    if (rc != WINO_OK) return rc;
+    pl->last_uq = Uq;
+    pl->last_ws = ws;
+    pl->last_stream = st;
+    return WINO_OK;
+  }
   // calibration on a single-kernel plan runs the staged kernels (dp4a or tcgen05 middle stage)
   const int saved_path = pl->path;
   int gemm_path = pl->path;
   if (pl->path == WINO_PATH_SMALLC) gemm_path = WINO_PATH_STAGED_DP4A;
   if (pl->path == WINO_PATH_FUSED_F2) gemm_path = WINO_PATH_STAGED_TC_PTR;
-  const bool tma_ok = pl->path == WINO_PATH_STAGED_TC && !calib;
+  if (pl->path == WINO_PATH_FUSED_LAYER) gemm_path = WINO_PATH_STAGED_TC;
+  const bool tma_ok = (pl->path == WINO_PATH_STAGED_TC || pl->path == WINO_PATH_STAGED_TC_MMA) && !calib;
+  const bool mma_ok = pl->path == WINO_PATH_STAGED_TC_MMA && !calib;
   int rc = WINO_OK;
   if (!(stage_mask & 1)) {
-  } else if (pl->launches++, tma_ok && pl->p.z_x == 0 && tma_chunk(pl->p.C) != 0) {
+  } else if (pl->launches++, mma_ok && pl->p.z_x == 0 &&
+             transform_mma_supported(pl->p, pl->std_mats, pl->p.C)) {
+    const CUtensorMap* mx = map_x_sw(pl, x);
+    const CUtensorMap* mv = map_stage(pl, pl->cache_vst, Vq, pl->p.C);
+    if (mx == nullptr || mv == nullptr) return WINO_ERR_CUDA;
+    rc = launch_input_transform_mma(pl->p, opt_of(pl, pdl), *mx, *mv, pl->kron_dev, pl->num_sms,
+                                    pl->status_dev, st);
+  } else if (tma_ok && pl->p.z_x == 0 && tma_chunk(pl->p.C) != 0) {
     const CUtensorMap* mx = map_x(pl, x);
     const CUtensorMap* mv = map_stage(pl, pl->cache_vst, Vq, pl->p.C);
     if (mx == nullptr || mv == nullptr) return WINO_ERR_CUDA;
@@ -302,7 +380,14 @@ int forward_impl(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float
   }
   if (rc != WINO_OK) return rc;
   if (!(stage_mask & 4)) {
-  } else if (pl->launches++, tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
+  } else if (pl->launches++, mma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 &&
+             transform_mma_supported(pl->p, pl->std_mats, pl->p.K)) {
+    const CUtensorMap* mm = map_m_sw(pl, mbuf);
+    const CUtensorMap* my = map_y(pl, y);
+    if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
+    rc = launch_output_transform_mma(pl->p, opt_of(pl, pdl), *mm, *my, pl->kron_dev, bias, pl->s_Y,
+                                     pl->num_sms, pl->status_dev, st);
+  } else if (tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
     const CUtensorMap* mm = map_stage(pl, pl->cache_mld, mbuf, pl->p.K);
     const CUtensorMap* my = map_y(pl, y);
     if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
@@ -402,8 +487,20 @@ int wino_plan(const wino_desc_t* desc, wino_plan_t** out) {
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, pl->device) == cudaSuccess &&
         sms > 0)
       pl->num_sms = sms;
-    if (cudaMalloc(&pl->status_dev, 256) == cudaSuccess) {
-      cudaMemset(pl->status_dev, 0, 256);
+    // one small allocation: the status word, then (256 bytes in) the Kronecker tables
+    const size_t dev_bytes = 256 + kKronBytes + sizeof(unsigned) * kFusedCounterWords;
+    if (cudaMalloc(&pl->status_dev, dev_bytes) == cudaSuccess) {
+      cudaMemset(pl->status_dev, 0, dev_bytes);
+      pl->kron_dev = reinterpret_cast<uint8_t*>(pl->status_dev) + 256;
+      pl->counters_dev = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(pl->kron_dev) + kKronBytes);
+      if (pl->std_mats && (d.m == 2 || d.m == 4)) {
+        int8_t tables[kKronBytes];
+        fill_kronecker_tables(d.m, tables);
+        if (cudaMemcpy(pl->kron_dev, tables, kKronBytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+          cudaFree(pl->status_dev);
+          pl->status_dev = nullptr;
+        }
+      }
     } else {
       pl->status_dev = nullptr;
     }
@@ -427,7 +524,7 @@ int wino_plan_path(const wino_plan_t* pl) { return pl ? pl->path : WINO_ERR_INVA
 
 int wino_plan_force_path(wino_plan_t* pl, int path) {
   if (pl == nullptr) return WINO_ERR_INVALID;
-  if (path < WINO_PATH_STAGED_TC || path > WINO_PATH_FUSED_F2) return WINO_ERR_INVALID;
+  if (path < WINO_PATH_STAGED_TC || path > WINO_PATH_FUSED_LAYER) return WINO_ERR_INVALID;
   if (!path_supported(pl, path)) return WINO_ERR_UNSUPPORTED;
   pl->path = path;
   return WINO_OK;
@@ -578,6 +675,7 @@ int wino_debug_dump_stage(wino_plan_t* pl, int stage, void* dst, size_t bytes) {
     const int saved_path = pl->path;
     if (pl->path == WINO_PATH_SMALLC) pl->path = WINO_PATH_STAGED_DP4A;
     if (pl->path == WINO_PATH_FUSED_F2) pl->path = WINO_PATH_STAGED_TC_PTR;
+    if (pl->path == WINO_PATH_FUSED_LAYER) pl->path = WINO_PATH_STAGED_TC;
     const int rc = launch_gemm(pl, reinterpret_cast<const int8_t*>(ws), pl->last_uq, dst, kOutI32,
                                nullptr, false, st);
     pl->path = saved_path;

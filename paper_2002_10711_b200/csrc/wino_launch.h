@@ -73,6 +73,35 @@ int launch_output_transform_tma(const Params& p, const LaunchOpt& o, const CUten
                                 const CUtensorMap& mapY, const float* bias, float s_Y, int* status,
                                 cudaStream_t st);
 
+// Tensor-core transforms (Cook-Toom F2 / F4, channel count a multiple of 128; input
+// needs z_x == 0, output needs Q_M on and an int8 output).  mapX and mapM carry the
+// 128-byte swizzle; mapV and mapY are the plain maps of the kernels above.
+// `kron`: device copy of the plan's Kronecker tables (fill_kronecker_tables).
+constexpr int kKronInRows = 48, kKronOutRows = 16;
+constexpr int kKronBytes = (kKronInRows + kKronOutRows) * 64;
+bool transform_mma_supported(const Params& p, bool std_mats, int channels);
+void fill_kronecker_tables(int m, int8_t* dst_host);
+int launch_input_transform_mma(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX,
+                               const CUtensorMap& mapV, const void* kron, int num_sms, int* status,
+                               cudaStream_t st);
+int launch_output_transform_mma(const Params& p, const LaunchOpt& o, const CUtensorMap& mapM,
+                                const CUtensorMap& mapY, const void* kron, const float* bias,
+                                float s_Y, int num_sms, int* status, cudaStream_t st);
+
+// The whole layer in one persistent launch (Cook-Toom F2 / F4, C and K multiples of
+// 128, input zero point 0, Q_M on, int8 output).  `counters`: plan-owned device words,
+// zero between launches (the kernel clears them when it finishes):
+// [kFusedMaxMblk] cnt_in, [kFusedMaxMblk] cnt_m, then the exit ticket.
+constexpr int kFusedMaxMblk = 1024;
+constexpr int kFusedCounterWords = 2 * kFusedMaxMblk + 16;
+struct FusedGeom { int BN, stages, n_mblk, n_nblk, n_items, grid; size_t smem; };
+struct FusedMaps { const CUtensorMap *x, *v_store, *v_load, *u, *m_load, *y; };
+bool layer_fused_supported(const Params& p, bool std_mats);
+FusedGeom layer_fused_geometry(const Params& p, int num_sms);
+int launch_layer_fused(const Params& p, const LaunchOpt& o, const FusedGeom& g, const FusedMaps& m,
+                       const void* kron, unsigned* counters, int8_t* mq, const float* bias,
+                       float s_Y, int* status, cudaStream_t st);
+
 struct TcGeom { int BN, MB, stages, tmem_cols, grid; size_t smem; };
 TcGeom tc_geometry(const Params& p, int num_sms);
 int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,

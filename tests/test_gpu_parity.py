@@ -13,7 +13,7 @@ from helpers import build_layer, small
 
 pytestmark = pytest.mark.gpu
 
-TC, DP4A, SMALLC, TC_PTR, FUSED = 1, 2, 3, 4, 5
+TC, DP4A, SMALLC, TC_PTR, FUSED, TC_MMA, LAYER = 1, 2, 3, 4, 5, 6, 7
 
 
 def _compare(L, x_q, w_q, bias, path, dumps=True):
@@ -49,12 +49,14 @@ SHAPES = [
     (2, 128, 9, 10, 192),    # TMA-staged transforms: 128- and 64-channel chunks, ragged tiles
     (1, 512, 4, 4, 512),     # 256-channel chunks, two per tile
     (3, 256, 7, 7, 128),     # odd tile count: last block of a 2-tile group is partial
+    (37, 128, 9, 9, 256),    # tensor-core transforms: more units than resident blocks, ragged tiles
+    (4, 384, 8, 8, 384),     # three 128-channel stages; the second 256-wide column block is half empty
 ]
 
 
 @pytest.mark.parametrize("m", [2, 4, 6])
 @pytest.mark.parametrize("shape", SHAPES)
-@pytest.mark.parametrize("path", [TC, TC_PTR, DP4A])
+@pytest.mark.parametrize("path", [TC, TC_MMA, TC_PTR, DP4A])
 def test_staged_paths_every_stage(m, shape, path):
     N, C, H, W, K = shape
     wl = wi.Workload("s", 3000 + m, N, C, H, W, K, m)
@@ -102,6 +104,75 @@ def test_small_channel_path(m, shape):
     L, x_q, w_q, bias = build_layer(wl)
     _compare(L, x_q, w_q, bias, SMALLC, dumps=False)
     _compare(L, x_q, w_q, bias, DP4A, dumps=True)
+
+
+LAYER_SHAPES = [
+    # N, C, H, W, K  (C and K multiples of 128)
+    (1, 128, 8, 8, 128),      # a handful of tiles: most CTAs have nothing to do
+    (2, 128, 9, 10, 256),     # ragged tiles
+    (37, 128, 9, 9, 256),     # several 128-tile blocks, the last one partial
+    (1, 512, 4, 4, 512),      # four channel chunks, two 256-wide column blocks
+    (3, 256, 7, 7, 128),
+    (16, 384, 8, 8, 384),     # second column block half empty
+    (60, 128, 16, 16, 128),   # many blocks of tiles: every CTA loops in all three phases
+]
+
+
+@pytest.mark.parametrize("m", [2, 4])
+@pytest.mark.parametrize("shape", LAYER_SHAPES)
+def test_single_launch_layer_every_stage(m, shape):
+    N, C, H, W, K = shape
+    wl = wi.Workload("l", 3900 + m, N, C, H, W, K, m)
+    L, x_q, w_q, bias = build_layer(wl)
+    g = _compare(L, x_q, w_q, bias, LAYER)
+    assert g["launches"] == 2          # weight transform + one launch for the whole layer
+
+
+@pytest.mark.parametrize("variant", ["relu", "no_bias", "zero_points_w_y", "saturating"])
+def test_single_launch_layer_variants(variant):
+    wl = wi.Workload("lv", 3950, 5, 256, 8, 10, 128, 4)
+    kw = {}
+    if variant == "relu":
+        kw["relu"] = True
+    if variant == "no_bias":
+        kw["with_bias"] = False
+    L, x_q, w_q, bias = build_layer(wl, **kw)
+    if variant == "zero_points_w_y":
+        L.q_w.zero_point = -3
+        L.q_Y.zero_point = 7
+    if variant == "saturating":
+        for q in (L.q_V, L.q_U, L.q_M, L.q_Y):
+            q.scale = q.scale / 7.0
+    _compare(L, x_q, w_q, bias, LAYER)
+
+
+def test_single_launch_layer_back_to_back_calls_reuse_the_counters():
+    import torch
+    from paper_2002_10711_b200 import binding
+    from paper_2002_10711_b200.layer import WinogradConv
+    wl = wi.Workload("lb", 3960, 9, 128, 8, 8, 256, 4)
+    L, x_q, w_q, bias = build_layer(wl)
+    y_ref = oracle.forward(L, x_q, w_q, bias=bias)
+    plan = binding.Plan.from_layer(L, path=LAYER)
+    conv = WinogradConv(plan)
+    conv.load_weights(w_q, bias)
+    x = torch.from_numpy(x_q).cuda()
+    ys = [conv.forward(x, conv.empty_output().fill_(0)) for _ in range(5)]
+    assert plan.last_status() == 0
+    for y in ys:
+        assert (y.cpu().numpy() == y_ref).all()
+
+
+def test_single_launch_layer_refuses_other_layers():
+    from paper_2002_10711_b200 import binding
+    for m, C, K, flex, kw in ((6, 128, 128, False, {}), (4, 64, 128, False, {}), (4, 128, 192, False, {}),
+                              (4, 128, 128, True, {}), (4, 128, 128, False, {"out_dtype": 1}),
+                              (4, 128, 128, False, {"q_M": False})):
+        wl = wi.Workload("lr", 3970, 1, C, 8, 8, K, m, flex=flex)
+        L, x_q, w_q, bias = build_layer(wl, **kw)
+        with pytest.raises(binding.WinoError) as e:
+            binding.Plan.from_layer(L, path=LAYER)
+        assert e.value.code == binding.ERR_UNSUPPORTED
 
 
 FUSED_SHAPES = [
@@ -178,6 +249,9 @@ def test_full_size_configs(name):
     L, x_q, w_q, bias = build_layer(wl)
     g = _compare(L, x_q, w_q, bias, TC)
     assert g["launches"] >= 4
+    _compare(L, x_q, w_q, bias, TC_MMA)
+    if name == "cfg3":
+        _compare(L, x_q, w_q, bias, LAYER)
     _compare(L, x_q, w_q, bias, TC_PTR)
     if name == "cfg2":
         _compare(L, x_q, w_q, bias, FUSED, dumps=False)
