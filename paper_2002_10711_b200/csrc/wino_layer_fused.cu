@@ -12,20 +12,30 @@
 // items.  The phases of different CTAs are tied together by counters in global
 // memory, one pair per block of 128 tiles ("m-block"):
 //   cnt_in[mb]  input-transform units of the m-block whose V_q is stored and visible;
-//   cnt_m[mb]   epilogue warps that have stored their share of an item of the m-block.
+//   cnt_m[mb]   16 per GEMM item of the m-block whose m_q is stored and visible.
 // A GEMM item waits for cnt_in of its m-block, an output unit for cnt_m of its
 // m-block; nothing in phase A waits for another CTA, so the dependency graph has
 // no cycle as long as every CTA is resident (the grid is at most one CTA per SM).
 // Every wait is bounded; on expiry the kernel records WINO_ERR_TIMEOUT and unwinds.
 // The last CTA to finish clears the counters for the next launch.
 //
-// Warp roles (640 threads):
-//   warp 0   TMA loads of the transform units (x patches, later m_q blocks)
-//   warp 1   transform MMAs (one lane)
+// Warp roles (800 threads):
+//   warp 0   TMA loads of the transform units (x patches, later m_q blocks), one lane
+//            per shared-memory slot; the other lanes prefetch x into L2
+//   warp 1   transform MMAs, one lane per worker group
 //   warp 2   TMA loads of the GEMM operands (U_q, V_q)
 //   warp 3   GEMM MMAs (one lane); owns the tensor-memory allocation
-//   warps 4-19  four worker groups of four warps (one per tensor-memory lane
+//   warp 4   publisher of cnt_m
+//   warps 5-8   one store thread per worker group: TMA stores of the group's staging
+//            tile (V_q, later y) and the cnt_in updates.  A store needs the better
+//            part of a microsecond to be complete and visible device-wide; these
+//            threads, which no arithmetic waits for, pay for that.
+//   warps 9-24  four worker groups of four warps (one per tensor-memory lane
 //            quadrant): epilogues of A, B and C, in that order.
+// A unit's position jj in the CTA's list (A units first, then C units) fixes its worker
+// group (jj % 4) and its shared-memory slot (jj % 8), so a slot and an accumulator are
+// always reused by the same lanes in program order: no waiter is ever more than one
+// barrier phase behind what it waits for.
 // While the workers are still quantizing phase A, warps 2 and 3 already run the
 // first GEMM item of the CTA into tensor-memory columns 0..255; the transform
 // accumulators live in columns 256..511 until phase A is done.
@@ -36,8 +46,10 @@ namespace wino {
 
 namespace {
 
-constexpr int kFlThreads = 640;
-constexpr int kSlots = 6;            // transform units in flight per CTA
+constexpr int kFlThreads = 800;
+constexpr int kFlWorker0 = 288;      // first worker thread
+constexpr int kSlots = 8;            // transform units in flight per CTA (a multiple of 4)
+constexpr int kPrefetchUnits = 96;   // units whose input is requested into L2 at the start
 constexpr long long kFlagWaitCycles = 600000000ll;   // ~0.3 s
 
 __device__ __forceinline__ uint64_t fl_desc_kmajor_sw64(uint32_t a) {
@@ -70,14 +82,6 @@ __device__ __forceinline__ void fl_tmem_ld4(uint32_t taddr, uint32_t (&r)[4]) {
                : "r"(taddr)
                : "memory");
 }
-template <int N>
-__device__ __forceinline__ void fl_bulk_wait_n() {       // all but the N newest groups complete
-  asm volatile("cp.async.bulk.wait_group %0;" ::"n"(N) : "memory");
-}
-template <int N>
-__device__ __forceinline__ void fl_bulk_wait_read_n() {
-  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
-}
 __device__ __forceinline__ void group_barrier(int g) {
   asm volatile("bar.sync %0, 128;" ::"r"(g + 1) : "memory");
 }
@@ -89,11 +93,11 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-// Publish: everything this thread has observed as complete becomes visible to a
-// thread that reads the counter with acquire semantics.
-__device__ __forceinline__ void flag_add(unsigned* p) {
-  fence_async_global();
-  asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
+// Counter update.  Relaxed on purpose: the updating thread issues ONE __threadfence()
+// before its updates (fence + relaxed write = release) instead of paying for a fence
+// inside every update (a release update costs ~1500 cycles each).
+__device__ __forceinline__ void flag_add(unsigned* p, unsigned v) {
+  asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 // Bounded wait for *p >= target; then order the acquire before later TMA reads.
 __device__ __forceinline__ bool flag_wait(const unsigned* p, unsigned target,
@@ -102,7 +106,7 @@ __device__ __forceinline__ bool flag_wait(const unsigned* p, unsigned target,
     const long long t0 = clock64();
     for (uint32_t i = 1;; ++i) {
       if (ld_acquire(p) >= target) break;
-      __nanosleep(i > 16u ? 200u : 40u);
+      __nanosleep(20u);
       if ((i & 63u) == 0u) {
         if (*abort_flag != 0u) return false;
         if (clock64() - t0 > kFlagWaitCycles) return false;
@@ -112,6 +116,37 @@ __device__ __forceinline__ bool flag_wait(const unsigned* p, unsigned target,
   fence_async_global();
   return true;
 }
+// Progress counter in shared memory (workers -> publisher).
+__device__ __forceinline__ void smem_count_add(uint32_t addr) {
+  asm volatile("red.release.cta.shared::cta.add.u32 [%0], 1;" ::"r"(addr) : "memory");
+}
+__device__ __forceinline__ uint32_t smem_count_read(uint32_t addr) {
+  uint32_t v;
+  asm volatile("ld.acquire.cta.shared::cta.u32 %0, [%1];" : "=r"(v) : "r"(addr) : "memory");
+  return v;
+}
+__device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int c0, int c1, int c2, int c3) {
+  asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+// Optional time stamps and failure codes (build with -DWINO_TRACE): 16 slots per CTA.
+#ifdef WINO_TRACE
+__device__ unsigned long long g_trace[256 * 16];
+__device__ long long g_trace_clk[256 * 16];
+__device__ __forceinline__ void trace(int slot) {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  g_trace[blockIdx.x * 16 + slot] = t;
+}
+#define WINO_TRACE_AT(slot) trace(slot)
+#define WINO_CLK_AT(cond, slot) do { if (cond) g_trace_clk[blockIdx.x * 16 + (slot)] = clock64(); } while (0)
+#define WINO_FAIL(code) atomicCAS((unsigned long long*)&g_trace_clk[blockIdx.x * 16 + 15], 0ull, (unsigned long long)(code))
+#else
+#define WINO_TRACE_AT(slot) ((void)0)
+#define WINO_CLK_AT(cond, slot) ((void)0)
+#define WINO_FAIL(code) ((void)0)
+#endif
 
 struct FusedArgs {
   int BN;             // GEMM block width (128 or 256)
@@ -122,6 +157,9 @@ struct FusedArgs {
   unsigned* cnt_m;    // [n_mblk]
   unsigned* ticket;   // CTAs that have finished
 };
+
+// Positions jj < n of a CTA's unit list that fall to group g (jj % 4 == g).
+__device__ __forceinline__ int group_units(int n, int g) { return n > g ? (n - g + 3) >> 2 : 0; }
 
 }  // namespace
 
@@ -137,8 +175,11 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
   constexpr int KROWS = (T2 + 31) / 32 * 32;          // transform MMA K: 32 (F2) or 64 (F4)
   constexpr int NB_IN = (T2 + 15) / 16 * 16;          // transform MMA N, input side: 16 or 48
   constexpr int NB_OUT = 16;
-  constexpr uint32_t kSlotBytes = KROWS * 128;
-  constexpr uint32_t kStageOut = T2 * 128;             // staging tile (input side is the larger)
+  // a slot holds the t*t rows TMA writes; the MMA reads KROWS rows, running into the next
+  // slot (or the pad behind the last one), where the Kronecker matrix has zero columns
+  constexpr uint32_t kSlotBytes = (T2 * 128 + 1023) / 1024 * 1024;
+  constexpr uint32_t kSlotRegion = kSlots * kSlotBytes + (KROWS * 128 - kSlotBytes);
+  constexpr uint32_t kStageOut = T2 * 128;             // staging tile, one per worker group
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
@@ -146,10 +187,10 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
   const uint32_t a_bytes = kBM * kStageK, b_bytes = (uint32_t)a.BN * kStageK;
   const uint32_t stage_bytes = a_bytes + b_bytes;
   const uint32_t s_ring = base;
-  const uint32_t s_slots = s_ring + (uint32_t)a.stages * stage_bytes;   // kSlots x kSlotBytes
-  const uint32_t s_kron = s_slots + kSlots * kSlotBytes;                // 64 rows x 64 B
-  const uint32_t s_stage = s_kron + 4096u;                              // 4 groups x 2 x kStageOut
-  const uint32_t s_bias = s_stage + 8u * kStageOut;                     // K floats (<= 1040)
+  const uint32_t s_slots = s_ring + (uint32_t)a.stages * stage_bytes;
+  const uint32_t s_kron = s_slots + kSlotRegion;                        // 64 rows x 64 B
+  const uint32_t s_stage = s_kron + 4096u;                              // 4 groups x kStageOut
+  const uint32_t s_bias = s_stage + 4u * kStageOut;                     // K floats (<= 1040)
   const uint32_t s_bar = s_bias + 4224u;
   const uint32_t bar_full = s_bar;                        // stages (<= 8)
   const uint32_t bar_empty = bar_full + 64u;
@@ -159,12 +200,19 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
   const uint32_t bar_tin_empty = bar_tin_full + 8u * kSlots;
   const uint32_t bar_tacc_full = bar_tin_empty + 8u * kSlots;   // 4
   const uint32_t bar_tacc_empty = bar_tacc_full + 32u;          // 4
-  const uint32_t bar_tr_done = bar_tacc_empty + 32u;            // 1
+  const uint32_t bar_st_full = bar_tacc_empty + 32u;            // 4 staging tiles
+  const uint32_t bar_st_empty = bar_st_full + 32u;              // 4
+  const uint32_t bar_kron = bar_st_empty + 32u;                 // 1: Kronecker tables are in place
+  const uint32_t bar_drain = bar_kron + 8u;                     // 5: last MMAs of an issuing thread are done
+  const uint32_t bar_tr_done = bar_drain + 40u;                 // 1
   const uint32_t bar_gemm_done = bar_tr_done + 8u;              // 1
-  const uint32_t tmem_slot = bar_gemm_done + 8u;
+  const uint32_t cnt_items = bar_gemm_done + 8u;                // u32: warps done with a GEMM item
+  const uint32_t tmem_slot = cnt_items + 8u;
   const uint32_t abort_slot = tmem_slot + 4u;
+  const uint32_t zero_slot = abort_slot + 4u;             // stays 0: "no abort" for the final drains
   volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
   volatile uint32_t* abort_p = reinterpret_cast<volatile uint32_t*>(gen + (abort_slot - base));
+  volatile uint32_t* zero_p = reinterpret_cast<volatile uint32_t*>(gen + (zero_slot - base));
   float* bias_s = reinterpret_cast<float*>(gen + (s_bias - base));
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -174,11 +222,13 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
   const int nA = cta < a.units_a ? (a.units_a - 1 - cta) / grid + 1 : 0;
   const int nC = cta < a.units_c ? (a.units_c - 1 - cta) / grid + 1 : 0;
   const int nI = cta < a.n_items ? (a.n_items - 1 - cta) / grid + 1 : 0;
+  const int nU = nA + nC;                               // the CTA's unit list: A units, then C units
   const int per_mb = T2 * a.n_nblk;                     // items per m-block
   const int cbuf = nI & 1;                              // GEMM accumulator buffer phase C borrows
 
   griddep_launch();
   if (threadIdx.x == 0) {
+    WINO_TRACE_AT(0);
     for (int s = 0; s < a.stages; ++s) {
       mbar_init(bar_full + 8u * s, 1);
       mbar_init(bar_empty + 8u * s, 1);
@@ -194,17 +244,18 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
     for (int g = 0; g < 4; ++g) {
       mbar_init(bar_tacc_full + 8u * g, 1);
       mbar_init(bar_tacc_empty + 8u * g, 4);
+      mbar_init(bar_st_full + 8u * g, 4);
+      mbar_init(bar_st_empty + 8u * g, 1);
     }
+    mbar_init(bar_kron, 16);
+    for (int i = 0; i < 5; ++i) mbar_init(bar_drain + 8u * i, 1);
     mbar_init(bar_tr_done, 16);
     mbar_init(bar_gemm_done, 16);
+    *reinterpret_cast<volatile uint32_t*>(gen + (cnt_items - base)) = 0u;
     *abort_p = 0u;
+    *zero_p = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  // Kronecker tables (plan constants): rows 0..47 input side, 48..63 output side
-  for (int idx = threadIdx.x; idx < 64 * 4; idx += kFlThreads)
-    *reinterpret_cast<uint4*>(gen + (s_kron - base) + fl_sw64_off(idx >> 2, (idx & 3) * 16)) =
-        __ldg(kron + idx);
-  fence_async_smem();
   if (warp == 3) tmem_alloc(tmem_slot, 512u);
   tc_fence_before();
   __syncthreads();
@@ -213,66 +264,110 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
 
   if (warp == 0) {
     // =============== transform loads: x patches (A), then m_q blocks (C) ===============
+    // Lane l owns slot l and loads every kSlots-th unit: a lone thread spends hundreds of
+    // cycles per unit on coordinates and issue, the lanes share that cost.  The lanes never
+    // block inside the loop (a lane spinning in a wait would hold the others at the warp's
+    // reconvergence point, and what it waits for may depend on them): each pass they test
+    // their conditions once and issue if everything is ready.
     if (lane == 0) {
       tma_prefetch_map(&mapX);
       tma_prefetch_map(&mapMld);
-      griddep_wait();
-      bool ok = true;
-      for (int jj = 0; jj < nA + nC && ok; ++jj) {
-        const uint32_t sl = (uint32_t)(jj % kSlots);
-        if (jj >= kSlots &&
-            !mbar_wait(bar_tin_empty + 8u * sl, (uint32_t)(jj / kSlots - 1) & 1u, abort_p)) { ok = false; break; }
-        mbar_expect_tx(bar_tin_full + 8u * sl, (uint32_t)T2 * 128u);
-        if (jj < nA) {
-          const int u = cta + jj * grid;
-          const int tau = u / cchunks, c0 = (u - tau * cchunks) << 7;
-          const int tw = tau % p.TW;
-          const int th = (tau / p.TW) % p.TH;
-          const int n = tau / (p.TW * p.TH);
-          tma_load_4d(s_slots + sl * kSlotBytes, &mapX, bar_tin_full + 8u * sl, c0, tw * M - 1, th * M - 1, n);
-        } else {
-          const int u = cta + (jj - nA) * grid;
-          const int tau = u / kchunks, k0 = (u - tau * kchunks) << 7;
-          const int mb = tau >> 7;
-          if (!flag_wait(a.cnt_m + mb, (unsigned)(per_mb * 16), abort_p)) { ok = false; break; }
-          tma_load_3d(s_slots + sl * kSlotBytes, &mapMld, bar_tin_full + 8u * sl, k0, tau, 0);
+    }
+    griddep_wait();
+    if (lane == 0) WINO_TRACE_AT(1);
+    if (lane >= kSlots) {
+      // x comes from HBM: the idle lanes ask for the patches of the units beyond the first
+      // round to be brought into L2 now, so that the loads below find them there
+      for (int jj = lane; jj < nA && jj < kPrefetchUnits; jj += 32 - kSlots) {
+        const int u = cta + jj * grid;
+        const int tau = u / cchunks, c0 = (u - tau * cchunks) << 7;
+        const int tw = tau % p.TW;
+        const int th = (tau / p.TW) % p.TH;
+        const int n = tau / (p.TW * p.TH);
+        tma_prefetch_l2_4d(&mapX, c0, tw * M - 1, th * M - 1, n);
+      }
+    } else {
+      const uint32_t sl = (uint32_t)lane;
+      int jj = lane, it = 0;
+      const long long t0 = clock64();
+      uint32_t spins = 0;
+      while (jj < nU) {
+        bool ready = it == 0 || mbar_try_wait(bar_tin_empty + 8u * sl, (uint32_t)(it - 1) & 1u);
+        int tau = 0, c0 = 0;
+        if (ready) {
+          const bool in_a = jj < nA;
+          const int u = cta + (in_a ? jj : jj - nA) * grid;
+          const int chunks = in_a ? cchunks : kchunks;
+          tau = u / chunks;
+          c0 = (u - tau * chunks) << 7;
+          if (!in_a) ready = ld_acquire(a.cnt_m + (tau >> 7)) >= (unsigned)(per_mb * 16);
+        }
+        if (ready) {
+          mbar_expect_tx(bar_tin_full + 8u * sl, (uint32_t)T2 * 128u);
+          if (jj < nA) {
+            const int tw = tau % p.TW;
+            const int th = (tau / p.TW) % p.TH;
+            const int n = tau / (p.TW * p.TH);
+            tma_load_4d(s_slots + sl * kSlotBytes, &mapX, bar_tin_full + 8u * sl, c0, tw * M - 1, th * M - 1, n);
+          } else {
+            fence_async_global();     // the counter was read with acquire; order the TMA read after it
+            if (jj == nA) WINO_TRACE_AT(12);
+            tma_load_3d(s_slots + sl * kSlotBytes, &mapMld, bar_tin_full + 8u * sl, c0, tau, 0);
+          }
+          jj += kSlots;
+          ++it;
+        } else if ((++spins & 1023u) == 0u && (*abort_p != 0u || clock64() - t0 > kWaitCycles)) {
+          WINO_FAIL(300 + jj);
+          *abort_p = 1u;
+          break;
         }
       }
-      if (!ok) *abort_p = 1u;
     }
   } else if (warp == 1) {
-    // =============== transform MMAs ===============
-    if (lane == 0) {
+    // =============== transform MMAs: lane g issues for worker group g ===============
+    // (same rule as above: no lane blocks inside the loop)
+    if (lane < 4) {
+      const int g = lane;
       const uint32_t idesc_in = fl_idesc_a_mn(128, NB_IN), idesc_out = fl_idesc_a_mn(128, NB_OUT);
       const uint64_t db_in = fl_desc_kmajor_sw64(s_kron);
       const uint64_t db_out = fl_desc_kmajor_sw64(s_kron + 48u * 64u);
-      bool ok = true;
-      for (int jj = 0; jj < nA + nC && ok; ++jj) {
+      const int nG = group_units(nU, g);
+      const long long t0 = clock64();
+      uint32_t spins = 0;
+      int n = 0;                                  // n-th unit of group g = n-th use of its accumulator
+      bool kron_ok = false, gemm_ok = nI == 0;
+      while (n < nG) {
+        const int jj = g + 4 * n;                 // position in the CTA's unit list
         const bool ph_c = jj >= nA;
-        if (jj == nA && nI > 0) {
-          // phase C borrows the columns of a GEMM accumulator buffer: every item of this
-          // CTA must have been drained first.  (A parity wait on bar_acc_empty would not
-          // do: this thread gets here long before the items, more than one phase ahead.)
-          if (!mbar_wait(bar_gemm_done, 0u, abort_p)) { ok = false; break; }
-        }
         const uint32_t sl = (uint32_t)(jj % kSlots);
-        const int jl = ph_c ? jj - nA : jj;
-        const int g = jl & 3;
-        // how often group g's accumulator has been used before this unit
-        const uint32_t use = (uint32_t)(jl >> 2) + (ph_c && nA > g ? (uint32_t)((nA - g + 3) >> 2) : 0u);
-        if (!mbar_wait(bar_tin_full + 8u * sl, (uint32_t)(jj / kSlots) & 1u, abort_p)) { ok = false; break; }
-        if (!mbar_wait(bar_tacc_empty + 8u * g, (use & 1u) ^ 1u, abort_p)) { ok = false; break; }
-        tc_fence_after();
-        const uint32_t tcol = tmem_base + (uint32_t)((ph_c ? cbuf : 1) * 256 + g * 64);
-        const uint64_t da = fl_desc_mnmajor_sw128(s_slots + sl * kSlotBytes);
+        if (!kron_ok) kron_ok = mbar_try_wait(bar_kron, 0u);        // the workers have copied the tables
+        // phase C borrows the columns of a GEMM accumulator buffer: every item of this CTA
+        // must have been drained first (a one-phase barrier: no parity to get ahead of)
+        if (ph_c && !gemm_ok) gemm_ok = mbar_try_wait(bar_gemm_done, 0u);
+        const bool ready = kron_ok && (!ph_c || gemm_ok) &&
+                           mbar_try_wait(bar_tin_full + 8u * sl, (uint32_t)(n >> 1) & 1u) &&
+                           mbar_try_wait(bar_tacc_empty + 8u * g, ((uint32_t)n & 1u) ^ 1u);
+        if (ready) {
+          tc_fence_after();
+          const uint32_t tcol = tmem_base + (uint32_t)((ph_c ? cbuf : 1) * 256 + g * 64);
+          const uint64_t da = fl_desc_mnmajor_sw128(s_slots + sl * kSlotBytes);
 #pragma unroll
-        for (int ks = 0; ks < KROWS / 32; ++ks)
-          mma_i8(tcol, da + (uint64_t)(ks * 256), (ph_c ? db_out : db_in) + (uint64_t)(ks * 2),
-                 ph_c ? idesc_out : idesc_in, ks != 0 ? 1u : 0u);
-        mma_commit(bar_tin_empty + 8u * sl);
-        mma_commit(bar_tacc_full + 8u * g);
+          for (int ks = 0; ks < KROWS / 32; ++ks)
+            mma_i8(tcol, da + (uint64_t)(ks * 256), (ph_c ? db_out : db_in) + (uint64_t)(ks * 2),
+                   ph_c ? idesc_out : idesc_in, ks != 0 ? 1u : 0u);
+          mma_commit(bar_tin_empty + 8u * sl);
+          mma_commit(bar_tacc_full + 8u * g);
+          ++n;
+        } else if ((++spins & 1023u) == 0u && (*abort_p != 0u || clock64() - t0 > kWaitCycles)) {
+          WINO_FAIL(400 + n * 4 + g + (kron_ok ? 0 : 10000) + (ph_c && !gemm_ok ? 20000 : 0));
+          *abort_p = 1u;
+          break;
+        }
       }
-      if (!ok) *abort_p = 1u;
+      // leave only when every MMA this thread has issued is done (also on the abort path:
+      // tensor memory is freed at the end of the kernel)
+      mma_commit(bar_drain + 8u * (uint32_t)g);
+      (void)mbar_wait<false>(bar_drain + 8u * (uint32_t)g, 0u, zero_p);
     }
   } else if (warp == 2) {
     // =============== GEMM operand loads ===============
@@ -281,32 +376,34 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
       tma_prefetch_map(&mapU);
       bool ok = true;
       int s = 0; uint32_t ph = 0;
-      // U_q is a constant of the layer: the first item's weight tiles are fetched before the
-      // wait on the preceding kernel; the V_q halves of the same stages follow the counter
-      int pre = 0;
-      if (nI > 0) {
-        const int it = cta;
-        const int rem = it % per_mb, xi = rem / a.n_nblk, nb = rem % a.n_nblk;
-        pre = KB < a.stages ? KB : a.stages;
-        for (int kb = 0; kb < pre; ++kb) {
-          mbar_expect_tx(bar_full + 8u * kb, stage_bytes);
-          tma_load_3d(s_ring + (uint32_t)kb * stage_bytes + a_bytes, &mapU, bar_full + 8u * kb,
-                      kb * kStageK, nb * a.BN, xi);
-        }
-      }
-      griddep_wait();
+      bool waited = false;     // griddepcontrol.wait done (U_q, a constant, may be fetched before it)
       for (int li = 0; li < nI && ok; ++li) {
         const int it = cta + li * grid;
         const int mb = it / per_mb, rem = it - mb * per_mb;
         const int xi = rem / a.n_nblk, nb = rem - xi * a.n_nblk;
         const int tiles = min(kBM, p.T - mb * kBM);
-        if (!flag_wait(a.cnt_in + mb, (unsigned)(tiles * cchunks), abort_p)) { ok = false; break; }
+        // weight halves of as many stages as the ring can take now: no dependency on phase A
+        int armed = 0;
+        {
+          int s2 = s; uint32_t ph2 = ph;
+          for (int kb = 0; kb < KB && kb < a.stages; ++kb) {
+            if (!mbar_wait<false>(bar_empty + 8u * s2, ph2 ^ 1u, abort_p)) { WINO_FAIL(101); ok = false; break; }
+            mbar_expect_tx(bar_full + 8u * s2, stage_bytes);
+            tma_load_3d(s_ring + (uint32_t)s2 * stage_bytes + a_bytes, &mapU, bar_full + 8u * s2,
+                        kb * kStageK, nb * a.BN, xi);
+            armed = kb + 1;
+            if (++s2 == a.stages) { s2 = 0; ph2 ^= 1u; }
+          }
+          if (!ok) break;
+        }
+        if (!waited) { griddep_wait(); waited = true; }
+        if (!flag_wait(a.cnt_in + mb, (unsigned)(tiles * cchunks), abort_p)) { WINO_FAIL(102); ok = false; break; }
+        if (li == 0) WINO_TRACE_AT(8);
+        if (li == 1) WINO_TRACE_AT(9);
         for (int kb = 0; kb < KB; ++kb) {
           const uint32_t sa = s_ring + (uint32_t)s * stage_bytes;
-          if (li == 0 && kb < pre) {
-            // stage already armed and its U_q half in flight
-          } else {
-            if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
+          if (kb >= armed) {
+            if (!mbar_wait<false>(bar_empty + 8u * s, ph ^ 1u, abort_p)) { WINO_FAIL(103); ok = false; break; }
             mbar_expect_tx(bar_full + 8u * s, stage_bytes);
             tma_load_3d(sa + a_bytes, &mapU, bar_full + 8u * s, kb * kStageK, nb * a.BN, xi);
           }
@@ -314,6 +411,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
           if (++s == a.stages) { s = 0; ph ^= 1u; }
         }
       }
+      if (!waited) griddep_wait();
       if (!ok) *abort_p = 1u;
     }
   } else if (warp == 3) {
@@ -325,14 +423,16 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
       for (int li = 0; li < nI && ok; ++li) {
         const int buf = li & 1;
         const uint32_t aph = (uint32_t)(li >> 1) & 1u;
-        if (!mbar_wait(bar_acc_empty + 8u * buf, aph ^ 1u, abort_p)) { ok = false; break; }
+        if (!mbar_wait<false>(bar_acc_empty + 8u * buf, aph ^ 1u, abort_p)) { WINO_FAIL(104); ok = false; break; }
         // columns 256..511 hold the transform accumulators until phase A is over
-        if (li == 1 && !mbar_wait(bar_tr_done, 0u, abort_p)) { ok = false; break; }
+        if (li == 1 && !mbar_wait<false>(bar_tr_done, 0u, abort_p)) { WINO_FAIL(105); ok = false; break; }
         tc_fence_after();
         const uint32_t tacc = tmem_base + (uint32_t)(buf * 256);
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(bar_full + 8u * s, ph, abort_p)) { ok = false; break; }
+          if (!mbar_wait<false>(bar_full + 8u * s, ph, abort_p)) { WINO_FAIL(106); ok = false; break; }
           tc_fence_after();
+          if (kb == 0 && li == 0) WINO_TRACE_AT(10);
+          if (kb == 0 && li == 1) WINO_TRACE_AT(11);
           const uint32_t sa = s_ring + (uint32_t)s * stage_bytes;
           const uint64_t da = make_desc_sw128(sa), db = make_desc_sw128(sa + a_bytes);
 #pragma unroll
@@ -345,31 +445,127 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
         mma_commit(bar_acc_full + 8u * buf);
       }
       if (!ok) *abort_p = 1u;
+      mma_commit(bar_drain + 32u);     // leave only when every MMA issued here is done
+      (void)mbar_wait<false>(bar_drain + 32u, 0u, zero_p);
+    }
+  } else if (warp == 4) {
+    // =============== publisher of cnt_m ===============
+    // an item's m_q is in place once all 16 epilogue warps have stored their share; one
+    // fence covers every item that finished in the meantime (fence + relaxed update = release)
+    if (lane == 0) {
+      const long long t0 = clock64();
+      uint32_t spins = 0;
+      int pub = 0;
+      while (pub < nI) {
+        const int fin = (int)(smem_count_read(cnt_items) >> 4);
+        if (fin > pub) {
+          __threadfence();
+          fence_async_global();
+          for (; pub < fin; ++pub) flag_add(a.cnt_m + (cta + pub * grid) / per_mb, 16u);
+        } else if ((++spins & 255u) == 0u && (*abort_p != 0u || clock64() - t0 > kWaitCycles)) {
+          WINO_FAIL(500 + pub);
+          *abort_p = 1u;
+          break;
+        }
+      }
+    }
+  } else if (warp < 9) {
+    // =============== store thread of worker group g ===============
+    if (lane == 0) {
+      const int g = warp - 5;
+      tma_prefetch_map(&mapVst);
+      tma_prefetch_map(&mapY);
+      const int nG = group_units(nU, g);
+      const uint32_t st = s_stage + (uint32_t)g * kStageOut;
+      bool ok = true;
+      // cnt_in updates are batched: waiting for a store to complete and fencing costs about
+      // two unit times, so it is done once per four tiles (and at the end of phase A), while
+      // the staging tile is handed back as soon as the store has read it
+      int pend = 0, pend_mb[4];
+      auto flush = [&]() {
+        if (pend == 0) return;
+        bulk_wait_all();                           // the V_q bytes are in place
+        __threadfence();
+        fence_async_global();
+        for (int i = 0; i < pend; ++i) {
+          unsigned cnt = 1u;
+          while (i + 1 < pend && pend_mb[i + 1] == pend_mb[i]) { ++cnt; ++i; }
+          flag_add(a.cnt_in + pend_mb[i], cnt);
+        }
+        pend = 0;
+      };
+      for (int n = 0; n < nG; ++n) {               // n-th tile of this group
+        const int jj = g + 4 * n;
+        if (!mbar_wait<false>(bar_st_full + 8u * (uint32_t)g, (uint32_t)n & 1u, abort_p)) { WINO_FAIL(600 + n); ok = false; break; }
+        if (jj < nA) {
+          const int u = cta + jj * grid;
+          const int tau = u / cchunks, c0 = (u - tau * cchunks) << 7;
+          tma_store_3d(&mapVst, st, c0, tau, 0);
+          bulk_commit();
+          bulk_wait_read();                        // the staging tile may be refilled
+          mbar_arrive(bar_st_empty + 8u * (uint32_t)g);
+          pend_mb[pend++] = tau >> 7;
+          if (pend == 4 || jj + 4 >= nA) flush();
+          if (g == 0 && jj + 4 >= nA) WINO_TRACE_AT(13);
+        } else {
+          // y tile (pixels past the image edge are clipped by the TMA unit)
+          const int u = cta + (jj - nA) * grid;
+          const int tau = u / kchunks, k0 = (u - tau * kchunks) << 7;
+          const int tw = tau % p.TW;
+          const int th = (tau / p.TW) % p.TH;
+          const int n_img = tau / (p.TW * p.TH);
+          tma_store_4d(&mapY, st, k0, tw * M, th * M, n_img);
+          bulk_commit();
+          bulk_wait_read();
+          mbar_arrive(bar_st_empty + 8u * (uint32_t)g);
+        }
+      }
+      flush();
+      bulk_wait_all();
+      if (!ok) *abort_p = 1u;
     }
   } else {
     // =============== workers ===============
-    const int g = (warp - 4) >> 2;              // group
+    const int g = (warp - 9) >> 2;              // group
     const int quad = warp & 3;                  // tensor-memory lane quadrant
-    const int et = threadIdx.x - 128 - g * 128; // 0..127 inside the group
+    const int et = threadIdx.x - kFlWorker0 - g * 128;   // 0..127 inside the group
     const bool leader = et == 0;
     const uint32_t lane_off = (uint32_t)(quad * 32) << 16;
     const int ch = quad * 32 + lane;            // channel inside a 128-channel chunk / row inside an m-block
+    // Kronecker tables (plan constants): rows 0..47 input side, 48..63 output side
+    for (int idx = threadIdx.x - kFlWorker0; idx < 64 * 4; idx += kFlThreads - kFlWorker0)
+      *reinterpret_cast<uint4*>(gen + (s_kron - base) + fl_sw64_off(idx >> 2, (idx & 3) * 16)) =
+          __ldg(kron + idx);
+    fence_async_smem();
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_kron);
     griddep_wait();                             // bias may be the previous kernel's output
-    for (int k = threadIdx.x - 128; k < p.K; k += kFlThreads - 128)
+    for (int k = threadIdx.x - kFlWorker0; k < p.K; k += kFlThreads - kFlWorker0)
       bias_s[k] = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)s_Y) : 0.0f;
     asm volatile("bar.sync 5, 512;" ::: "memory");
-    uint32_t tuse = 0;                          // uses of this group's transform accumulator
+    const uint32_t st = s_stage + (uint32_t)g * kStageOut;
+    uint8_t* sp = gen + (st - base) + ch;       // this thread's column of the staging tile
+    uint32_t tuse = 0;                          // units this group has processed (A and C together)
+    int jj = g;                                 // position in the CTA's unit list
     bool ok = true;
+
+    // wait (every thread, bounded) until the store thread has read the previous tile out of
+    // the staging buffer; placed after the arithmetic, so it has normally long happened
+    auto staging_free = [&]() -> bool {
+      if (tuse == 0) return true;
+      return mbar_wait<false>(bar_st_empty + 8u * (uint32_t)g, (tuse & 1u) ^ 1u, abort_p);
+    };
 
     // ---------------- phase A ----------------
     {
       const float lo = __fadd_rn(p.lo_V, kMagic), hi = __fadd_rn(p.hi_V, kMagic);
-      int prev_mb = -1, jj = 0;
-      for (int j = g; j < nA; j += 4, ++jj, ++tuse) {
-        const int u = cta + j * grid;
-        const int tau = u / cchunks, c0 = (u - tau * cchunks) << 7;
-        if (leader && !mbar_wait(bar_tacc_full + 8u * g, tuse & 1u, abort_p)) *abort_p = 1u;
+      for (; jj < nA; jj += 4, ++tuse) {
+        WINO_CLK_AT(leader && g == 0 && tuse == 1, 0);
+        if (leader && !mbar_wait<false>(bar_tacc_full + 8u * g, tuse & 1u, abort_p)) { WINO_FAIL(201); *abort_p = 1u; }
+        if (leader && g == 0 && tuse == 0) WINO_TRACE_AT(2);
+        WINO_CLK_AT(leader && g == 0 && tuse == 1, 1);
         group_barrier(g);
+        WINO_CLK_AT(leader && g == 0 && tuse == 1, 2);
         if (*abort_p != 0u) { ok = false; break; }
         (void)mbar_try_wait(bar_tacc_full + 8u * g, tuse & 1u);
         tc_fence_after();
@@ -383,35 +579,34 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
           fl_tmem_ld16(tacc, r0);
         }
         tmem_ld_wait();
+        WINO_CLK_AT(leader && g == 0 && tuse == 1, 3);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tacc_empty + 8u * g);
-        const uint32_t st = s_stage + (uint32_t)(g * 2 + (jj & 1)) * kStageOut;
-        auto put = [&](int xi, uint32_t acc) {
-          const float r = fminf(fmaxf(__fmaf_rn(__int2float_rn((int)acc), p.mult_V, kMagic), lo), hi);
-          asm volatile("st.shared.u8 [%0], %1;" ::"r"(st + (uint32_t)(xi * 128 + ch)), "r"(__float_as_uint(r))
-                       : "memory");
+        // all codes first (independent chains the compiler can interleave), then the stores
+        auto code = [&](uint32_t acc) {
+          return __float_as_uint(fminf(fmaxf(__fmaf_rn(__int2float_rn((int)acc), p.mult_V, kMagic), lo), hi));
         };
 #pragma unroll
-        for (int q = 0; q < N0; ++q) put(q, r0[q]);
+        for (int q = 0; q < N0; ++q) r0[q] = code(r0[q]);
         if constexpr (M == 4) {
 #pragma unroll
-          for (int q = 0; q < N1; ++q) put(32 + q, r1[q]);
+          for (int q = 0; q < N1; ++q) r1[q] = code(r1[q]);
         }
+        if (!staging_free()) { WINO_FAIL(202); *abort_p = 1u; }
+#pragma unroll
+        for (int q = 0; q < N0; ++q) sp[q * 128] = (uint8_t)r0[q];
+        if constexpr (M == 4) {
+#pragma unroll
+          for (int q = 0; q < N1; ++q) sp[(32 + q) * 128] = (uint8_t)r1[q];
+        }
+        WINO_CLK_AT(leader && g == 0 && tuse == 1, 4);
         fence_async_smem();
-        group_barrier(g);
-        if (leader) {
-          tma_store_3d(&mapVst, st, c0, tau, 0);
-          bulk_commit();
-          fl_bulk_wait_n<1>();                  // the previous unit's store is complete
-          if (prev_mb >= 0) flag_add(a.cnt_in + prev_mb);
-          prev_mb = tau >> 7;
-        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_st_full + 8u * (uint32_t)g);   // the group's store thread takes over
+        WINO_CLK_AT(leader && g == 0 && tuse == 1, 5);
       }
-      if (leader) {
-        fl_bulk_wait_n<0>();
-        if (prev_mb >= 0) flag_add(a.cnt_in + prev_mb);
-      }
+      if (leader && g == 0) WINO_TRACE_AT(3);
       __syncwarp();
       if (lane == 0) mbar_arrive(bar_tr_done);
     }
@@ -425,12 +620,15 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
         const int xi = rem / a.n_nblk, nb = rem - xi * a.n_nblk;
         const int buf = li & 1;
         const uint32_t aph = (uint32_t)(li >> 1) & 1u;
-        if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8u * buf, aph, abort_p))) {
+        if (!__all_sync(0xffffffffu, mbar_wait<false>(bar_acc_full + 8u * buf, aph, abort_p))) {
+          WINO_FAIL(203);
           *abort_p = 1u;
           ok = false;
           break;
         }
         tc_fence_after();
+        if (leader && g == 0 && li == 0) WINO_TRACE_AT(4);
+        if (leader && g == 0 && li == 1) WINO_TRACE_AT(5);
         const uint32_t tacc = tmem_base + (uint32_t)(buf * 256) + lane_off;
         const int tau = mb * kBM + ch;
         for (int col = g * 32; col < a.BN; col += 128) {
@@ -440,42 +638,43 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
           tmem_ld_wait();
           const int k0 = nb * a.BN + col;
           if (tau < p.T && k0 < p.K) {
-          uint32_t w[8];
+            uint32_t w[8];
 #pragma unroll
-          for (int q = 0; q < 8; ++q) {
-            float f[4];
+            for (int q = 0; q < 8; ++q) {
+              float f[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
-              f[e] = fminf(fmaxf(__fmaf_rn(__int2float_rn((int)r[4 * q + e]), p.mult_M, kMagic), lo), hi);
-            const uint32_t l2 = __byte_perm(__float_as_uint(f[0]), __float_as_uint(f[1]), 0x0040u);
-            const uint32_t h2 = __byte_perm(__float_as_uint(f[2]), __float_as_uint(f[3]), 0x0040u);
-            w[q] = __byte_perm(l2, h2, 0x5410u);
-          }
-          uint4* dst = reinterpret_cast<uint4*>(mq + ((long)xi * p.T + tau) * p.K + k0);
-          dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-          dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+              for (int e = 0; e < 4; ++e)
+                f[e] = fminf(fmaxf(__fmaf_rn(__int2float_rn((int)r[4 * q + e]), p.mult_M, kMagic), lo), hi);
+              const uint32_t l2 = __byte_perm(__float_as_uint(f[0]), __float_as_uint(f[1]), 0x0040u);
+              const uint32_t h2 = __byte_perm(__float_as_uint(f[2]), __float_as_uint(f[3]), 0x0040u);
+              w[q] = __byte_perm(l2, h2, 0x5410u);
+            }
+            uint4* dst = reinterpret_cast<uint4*>(mq + ((long)xi * p.T + tau) * p.K + k0);
+            dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+            dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
           }
         }
         tc_fence_before();
         __syncwarp();
         if (lane == 0) {
           mbar_arrive(bar_acc_empty + 8u * buf);
-          __threadfence();
-          flag_add(a.cnt_m + mb);
+          smem_count_add(cnt_items);                 // release: this warp's m_q stores precede it
         }
       }
     }
-
+    if (leader && g == 0) WINO_TRACE_AT(6);
     __syncwarp();
     if (lane == 0) mbar_arrive(bar_gemm_done);
 
     // ---------------- phase C ----------------
     if (ok) {
-      int jj = 0;
-      for (int j = g; j < nC; j += 4, ++jj, ++tuse) {
-        const int u = cta + j * grid;
+      bool first = true;
+      for (; jj < nU; jj += 4, ++tuse) {
+        const int u = cta + (jj - nA) * grid;
         const int tau = u / kchunks, k0 = (u - tau * kchunks) << 7;
-        if (leader && !mbar_wait(bar_tacc_full + 8u * g, tuse & 1u, abort_p)) *abort_p = 1u;
+        if (leader && !mbar_wait<false>(bar_tacc_full + 8u * g, tuse & 1u, abort_p)) { WINO_FAIL(204); *abort_p = 1u; }
+        if (leader && g == 0 && first) WINO_TRACE_AT(7);
+        first = false;
         group_barrier(g);
         if (*abort_p != 0u) { ok = false; break; }
         (void)mbar_try_wait(bar_tacc_full + 8u * g, tuse & 1u);
@@ -487,26 +686,19 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
         __syncwarp();
         if (lane == 0) mbar_arrive(bar_tacc_empty + 8u * g);
         const float b_scaled = bias_s[k0 + ch];
-        const uint32_t st = s_stage + (uint32_t)(g * 2 + (jj & 1)) * kStageOut;
 #pragma unroll
         for (int q = 0; q < MM; ++q) {
           const float yf = __fmaf_rn(__int2float_rn((int)v[q]), p.mult_Y, b_scaled);
           const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
-          const uint32_t code = (uint32_t)(magic_to_int(r) + p.z_Y);
-          asm volatile("st.shared.u8 [%0], %1;" ::"r"(st + (uint32_t)(q * 128 + ch)), "r"(code) : "memory");
+          v[q] = (uint32_t)(magic_to_int(r) + p.z_Y);
         }
+        if (!staging_free()) { WINO_FAIL(205); *abort_p = 1u; }
+#pragma unroll
+        for (int q = 0; q < MM; ++q) sp[q * 128] = (uint8_t)v[q];
         fence_async_smem();
-        group_barrier(g);
-        if (leader) {
-          const int tw = tau % p.TW;
-          const int th = (tau / p.TW) % p.TH;
-          const int n = tau / (p.TW * p.TH);
-          tma_store_4d(&mapY, st, k0, tw * M, th * M, n);
-          bulk_commit();
-          fl_bulk_wait_read_n<1>();
-        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(bar_st_full + 8u * (uint32_t)g);
       }
-      if (leader) fl_bulk_wait_n<0>();
     }
     if (!ok) *abort_p = 1u;
   }
@@ -514,6 +706,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
   tc_fence_before();
   __syncthreads();
   if (threadIdx.x == 0) {
+    WINO_TRACE_AT(14);
     if (*abort_p != 0u) atomicExch(status, -6);  // WINO_ERR_TIMEOUT
     // the last CTA to get here clears the counters for the next launch
     __threadfence();
@@ -541,8 +734,10 @@ FusedGeom layer_fused_geometry(const Params& p, int num_sms) {
   FusedGeom g;
   g.BN = p.K >= 256 ? 256 : 128;
   const int t2 = p.t * p.t;
-  const size_t slot = (size_t)((t2 + 31) / 32 * 32) * 128;
-  const size_t fixed = 1024 + kSlots * slot + 4096 + 8 * (size_t)t2 * 128 + 4224 + 512;
+  const size_t krows = (size_t)(t2 + 31) / 32 * 32;
+  const size_t slot = ((size_t)t2 * 128 + 1023) / 1024 * 1024;
+  const size_t slot_region = kSlots * slot + (krows * 128 - slot);
+  const size_t fixed = 1024 + slot_region + 4096 + 4 * (size_t)t2 * 128 + 4224 + 640;
   const size_t stage = (size_t)kBM * kStageK + (size_t)g.BN * kStageK;
   int stages = (int)((227 * 1024 - fixed) / stage);
   if (stages > 8) stages = 8;
@@ -574,6 +769,15 @@ int fused_launch(const Params& p, const LaunchOpt& o, const FusedGeom& g, const 
                        reinterpret_cast<const uint4*>(kron), mq, bias, s_Y, status);
 }
 }  // namespace
+
+#ifdef WINO_TRACE
+extern "C" int wino_trace_read(unsigned long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_trace, sizeof(g_trace)) == cudaSuccess ? 0 : -5;
+}
+extern "C" int wino_trace_read_clk(long long* host_out) {
+  return cudaMemcpyFromSymbol(host_out, g_trace_clk, sizeof(g_trace_clk)) == cudaSuccess ? 0 : -5;
+}
+#endif
 
 int launch_layer_fused(const Params& p, const LaunchOpt& o, const FusedGeom& g, const FusedMaps& m,
                        const void* kron, unsigned* counters, int8_t* mq, const float* bias,

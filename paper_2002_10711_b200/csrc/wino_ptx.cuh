@@ -38,7 +38,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 // Bounded wait: polls until the phase completes, another role has raised the
 // abort flag, or about a second of SM clocks has passed.  On failure the caller
 // raises the abort flag and unwinds; the host reads WINO_ERR_TIMEOUT.
+// BACKOFF: sleep between polls (a spinning warp takes issue slots from the warps
+// it waits for).  Waits on the critical path of a pipeline poll without it: the
+// sleep's granularity is far coarser than the tens of cycles such a wait lasts.
 constexpr long long kWaitCycles = 2000000000ll;
+template <bool BACKOFF = true>
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
                                           volatile uint32_t* abort_flag,
                                           long long limit_cycles = kWaitCycles) {
@@ -46,8 +50,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
   const long long t0 = clock64();
   for (uint32_t i = 1;; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
-    // a spinning warp takes issue slots from the warps it waits for: back off
-    if (i > 8u) __nanosleep(i > 64u ? 128u : 32u);
+    if (BACKOFF && i > 8u) __nanosleep(i > 64u ? 128u : 32u);
     if ((i & 255u) == 0u) {
       if (*abort_flag != 0u) return false;
       if (clock64() - t0 > limit_cycles) return false;
