@@ -25,7 +25,7 @@
 //   warp 1   transform MMAs, one lane per worker group
 //   warp 2   TMA loads of the GEMM operands (U_q, V_q)
 //   warp 3   GEMM MMAs (one lane); owns the tensor-memory allocation
-//   warp 4   publisher of cnt_m
+//   warp 4   bias / s_Y table at the start, then publisher of cnt_m
 //   warps 5-8   one store thread per worker group: TMA stores of the group's staging
 //            tile (V_q, later y) and the cnt_in updates.  A store needs the better
 //            part of a microsecond to be complete and visible device-wide; these
@@ -204,7 +204,8 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
   const uint32_t bar_st_empty = bar_st_full + 32u;              // 4
   const uint32_t bar_kron = bar_st_empty + 32u;                 // 1: Kronecker tables are in place
   const uint32_t bar_drain = bar_kron + 8u;                     // 5: last MMAs of an issuing thread are done
-  const uint32_t bar_tr_done = bar_drain + 40u;                 // 1
+  const uint32_t bar_bias = bar_drain + 40u;                    // 1: bias table is in place
+  const uint32_t bar_tr_done = bar_bias + 8u;                   // 1
   const uint32_t bar_gemm_done = bar_tr_done + 8u;              // 1
   const uint32_t cnt_items = bar_gemm_done + 8u;                // u32: warps done with a GEMM item
   const uint32_t tmem_slot = cnt_items + 8u;
@@ -248,6 +249,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
       mbar_init(bar_st_empty + 8u * g, 1);
     }
     mbar_init(bar_kron, 16);
+    mbar_init(bar_bias, 1);
     for (int i = 0; i < 5; ++i) mbar_init(bar_drain + 8u * i, 1);
     mbar_init(bar_tr_done, 16);
     mbar_init(bar_gemm_done, 16);
@@ -449,7 +451,12 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
       (void)mbar_wait<false>(bar_drain + 32u, 0u, zero_p);
     }
   } else if (warp == 4) {
-    // =============== publisher of cnt_m ===============
+    // =============== bias table, then publisher of cnt_m ===============
+    griddep_wait();                             // bias may be the previous kernel's output
+    for (int k = lane; k < p.K; k += 32)
+      bias_s[k] = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)s_Y) : 0.0f;
+    __syncwarp();
+    if (lane == 0) mbar_arrive(bar_bias);
     // an item's m_q is in place once all 16 epilogue warps have stored their share; one
     // fence covers every item that finished in the meantime (fence + relaxed update = release)
     if (lane == 0) {
@@ -479,7 +486,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
       const uint32_t st = s_stage + (uint32_t)g * kStageOut;
       bool ok = true;
       // cnt_in updates are batched: waiting for a store to complete and fencing costs about
-      // two unit times, so it is done once per four tiles (and at the end of phase A), while
+      // two unit times, so it is done once per two tiles (and at the end of phase A), while
       // the staging tile is handed back as soon as the store has read it
       int pend = 0, pend_mb[4];
       auto flush = [&]() {
@@ -505,7 +512,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
           bulk_wait_read();                        // the staging tile may be refilled
           mbar_arrive(bar_st_empty + 8u * (uint32_t)g);
           pend_mb[pend++] = tau >> 7;
-          if (pend == 4 || jj + 4 >= nA) flush();
+          if (pend == 2 || jj + 4 >= nA) flush();
           if (g == 0 && jj + 4 >= nA) WINO_TRACE_AT(13);
         } else {
           // y tile (pixels past the image edge are clipped by the TMA unit)
@@ -521,7 +528,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
         }
       }
       flush();
-      bulk_wait_all();
+      bulk_wait_read();   // the y stores have read their tiles; the end of the grid publishes them
       if (!ok) *abort_p = 1u;
     }
   } else {
@@ -539,10 +546,6 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
     fence_async_smem();
     __syncwarp();
     if (lane == 0) mbar_arrive(bar_kron);
-    griddep_wait();                             // bias may be the previous kernel's output
-    for (int k = threadIdx.x - kFlWorker0; k < p.K; k += kFlThreads - kFlWorker0)
-      bias_s[k] = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)s_Y) : 0.0f;
-    asm volatile("bar.sync 5, 512;" ::: "memory");
     const uint32_t st = s_stage + (uint32_t)g * kStageOut;
     uint8_t* sp = gen + (st - base) + ch;       // this thread's column of the staging tile
     uint32_t tuse = 0;                          // units this group has processed (A and C together)
@@ -667,6 +670,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
     if (lane == 0) mbar_arrive(bar_gemm_done);
 
     // ---------------- phase C ----------------
+    if (ok && !mbar_wait<false>(bar_bias, 0u, abort_p)) { WINO_FAIL(206); ok = false; }
     if (ok) {
       bool first = true;
       for (; jj < nU; jj += 4, ++tuse) {
@@ -700,6 +704,7 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
         if (lane == 0) mbar_arrive(bar_st_full + 8u * (uint32_t)g);
       }
     }
+    if (leader && g == 0) WINO_TRACE_AT(15);
     if (!ok) *abort_p = 1u;
   }
   __syncwarp();
