@@ -33,11 +33,31 @@ if ROOT not in sys.path:
 
 import wino_inputs as wi  # noqa: E402
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu capture
-# of the cfg3 workload with the kernels as they stand; set an entry to None when its kernel
-# changes and the counters have not been taken again.
-NCU_TRAFFIC_CFG3 = {"k_input_transform_tma": 4.21e6, "k_gemm_tc": 11.84e6,
-                    "k_output_transform_tma": 9.45e6}
+PATH_NAMES = {1: "staged_tc", 2: "staged_dp4a", 3: "smallc", 4: "staged_tc_ptr", 5: "fused_f2",
+              6: "staged_tc_mma", 7: "fused_layer"}
+
+
+def csrc_digest():
+    """SHA-256 over the CUDA sources: identifies the kernels a profiler capture belongs to."""
+    import hashlib
+    root = os.path.join(ROOT, "paper_2002_10711_b200", "csrc")
+    h = hashlib.sha256()
+    for name in sorted(os.listdir(root)):
+        if name.endswith((".cu", ".cuh", ".h")):
+            h.update(name.encode())
+            h.update(open(os.path.join(root, name), "rb").read())
+    return h.hexdigest()
+
+
+def load_counters():
+    """profiles/traffic.json: per-kernel ncu counters of the cfg3 workload (DRAM bytes and
+    warp instructions per launch) with the digest of the sources they were taken from.
+    Returns {} when the sources have changed since (stale counters are not reported)."""
+    path = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(path):
+        return {}
+    d = json.load(open(path))
+    return d.get("kernels", {}) if d.get("csrc_sha256") == csrc_digest() else {}
 
 METRIC = "effective direct-conv-equivalent int8 TOPS (Winograd-aware quantized 3x3 conv forward)"
 UNIT = "TOPS"
@@ -168,6 +188,78 @@ def aggregate(ms_local: float, units_local: float, dist=None):
     return float(t.item()), float(u.item())
 
 
+def time_layer_quick(binding, cook_toom, torch, dev, N, C, H, W, K, m, flex_seed=None, path=0,
+                     steps=96):
+    """Steady-state microseconds per forward call of one layer shape on rotating buffers
+    (more bytes than L2), from a CUDA graph, with fixed stage scales: the kernels have no
+    data-dependent control flow, so for timing the values and scales do not matter.
+    Returns (us, path) or (None, reason)."""
+    BT, G, AT = cook_toom(m)
+    if flex_seed is not None:
+        BT = wi.flex_perturb(BT, flex_seed, wi.S_BT)
+        G = wi.flex_perturb(G, flex_seed, wi.S_G)
+        AT = wi.flex_perturb(AT, flex_seed, wi.S_AT)
+    q = lambda sc: dict(scale=sc)
+    try:
+        plan = binding.Plan(N, C, H, W, K, m, BT, G, AT, q(1 / 32), q(0.004), q(0.5), q(0.01),
+                            q(30.0), q(100.0), path=path)
+    except binding.WinoError as e:
+        return None, str(e)
+    xb, yb = N * H * W * C, N * H * W * K
+    R = max(2, int(np.ceil(1.5 * 126e6 / (xb + yb + plan.weight_bytes))))
+    gen = torch.Generator(device="cpu").manual_seed(7)
+    x0 = torch.randint(0, 127, (N, H, W, C), dtype=torch.int8, generator=gen).to(dev)
+    w = torch.randint(-127, 127, (K, 3, 3, C), dtype=torch.int8, generator=gen).to(dev)
+    xs = [x0.clone() for _ in range(R)]
+    ys = [torch.empty((N, H, W, K), dtype=torch.int8, device=dev) for _ in range(R)]
+    Us = [torch.empty(plan.weight_bytes, dtype=torch.int8, device=dev) for _ in range(R)]
+    ws = torch.empty(max(plan.workspace_bytes, 16), dtype=torch.uint8, device=dev)
+    for U in Us:
+        plan.transform_weights(w, U)
+
+    def step(i):
+        j = i % R
+        plan.conv_forward(xs[j], Us[j], None, ys[j], ws)
+
+    for i in range(3):
+        step(i)
+    torch.cuda.synchronize()
+    inner = max(2 * R, 8)
+    side = torch.cuda.Stream(device=dev)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            for i in range(inner):
+                step(i)
+    torch.cuda.synchronize()
+    g.replay()
+    torch.cuda.synchronize()
+    reps = max(1, steps // inner)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    if plan.last_status() != 0:
+        return None, "device status"
+    return e0.elapsed_time(e1) * 1e3 / (reps * inner), plan.path
+
+
+def layer_row(peaks, name, N, C, H, W, K, m, us, path):
+    t = m + 2
+    T = N * (-(-H // m)) * (-(-W // m))
+    d_ops = 2.0 * N * H * W * K * C * 9
+    w_ops = 2.0 * T * t * t * C * K
+    alg_bytes = N * H * W * (C + K) + t * t * K * C
+    roof = max(w_ops / (2.0 * peaks["bf16_tflops"] * 1e12), alg_bytes / (peaks["hbm_gbs"] * 1e9))
+    return {"layer": name, "N": N, "C": C, "K": K, "H": H, "W": W, "m": m,
+            "us": round(us, 2), "path": PATH_NAMES.get(path, str(path)),
+            "effective_TOPS": round(d_ops / (us * 1e-6) / 1e12, 1),
+            "wino_domain_TOPS": round(w_ops / (us * 1e-6) / 1e12, 1),
+            "roofline_us": round(roof * 1e6, 2), "frac": round(roof * 1e6 / us, 4)}
+
+
 def run_ours(args, wl):
     import torch
     import torch.distributed as dist
@@ -198,15 +290,15 @@ def run_ours(args, wl):
         AT = wi.flex_perturb(AT, wl.seed, wi.S_AT)
     q = lambda s, **kw: dict(scale=float(s), **kw)
 
-    def make_plan(s_V, s_U, s_M, s_Y):
+    def make_plan(s_V, s_U, s_M, s_Y, path=binding.PATH_AUTO):
         return binding.Plan(wl.N, wl.C, wl.H, wl.W, wl.K, wl.m, BT, G, AT, q(s_x), q(s_w), q(s_V),
-                            q(s_U), q(s_M), q(s_Y), out_dtype=0)
+                            q(s_U), q(s_M), q(s_Y), out_dtype=0, path=path)
 
     if wl.fixed_scales is not None:
         s_V = s_U = s_M = s_Y = float(np.float32(wl.fixed_scales))
     else:
         s_V, s_U, s_M, s_Y = calibrate(make_plan, x_q, w_q, bias, s_x, s_w, device=dev)
-    plan = make_plan(s_V, s_U, s_M, s_Y)
+    plan = make_plan(s_V, s_U, s_M, s_Y, path=args.path)
 
     # ---- device buffers: R rotating sets so that x, y and U_q come from HBM ----
     xb = x_q.nbytes
@@ -241,7 +333,7 @@ def run_ours(args, wl):
             for i in range(chunk):
                 step(i)
     torch.cuda.synchronize()
-    single_kernel = plan.path in (binding.PATH_SMALLC, binding.PATH_FUSED_F2)
+    single_kernel = plan.path in (binding.PATH_SMALLC, binding.PATH_FUSED_F2, binding.PATH_FUSED_LAYER)
     launches_per_step = 1 if single_kernel else 3
     graph.replay()
     torch.cuda.synchronize()
@@ -283,7 +375,8 @@ def run_ours(args, wl):
         # one fused kernel per step: its launch duration is the step time
         alg_bytes = xb + yb + plan.weight_bytes
         ach = alg_bytes / (ms_local / args.steps * 1e-3) / 1e9
-        roofline = {"kernel": "k_fused_f2" if plan.path == binding.PATH_FUSED_F2 else "k_smallc",
+        roofline = {"kernel": {binding.PATH_FUSED_F2: "k_fused_f2", binding.PATH_SMALLC: "k_smallc",
+                               binding.PATH_FUSED_LAYER: "k_layer_fused"}[plan.path],
                     "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                     "frac": ach / peaks["hbm_gbs"], "traffic": None,
                     "peak_note": f"of {peaks['source']}"}
@@ -326,21 +419,25 @@ def run_ours(args, wl):
                   for n, u in zip(names, us)}
         stages["hadamard_gemm"]["wino_TOPS"] = wino_ops(wl, wl.N) / (us[1] * 1e-6) / 1e12
         dom = max(range(3), key=lambda k: us[k])
-        kernel_names = {"input_transform": "k_input_transform_tma", "hadamard_gemm": "k_gemm_tc",
-                        "output_transform": "k_output_transform_tma"}
+        mma_tr = plan.path == binding.PATH_STAGED_TC_MMA
+        kernel_names = {"input_transform": "k_input_transform_mma" if mma_tr else "k_input_transform_tma",
+                        "hadamard_gemm": "k_gemm_tc",
+                        "output_transform": "k_output_transform_mma" if mma_tr else "k_output_transform_tma"}
+        counters = load_counters() if wl.name == "cfg3" else {}
+        traffic_of = lambda k: (counters.get(k) or {}).get("dram_bytes")
         if dom == 1:
             peak = 2.0 * peaks["bf16_tflops"]
             ach = wino_ops(wl, wl.N) / (us[1] * 1e-6) / 1e12
             roofline = {"kernel": "k_gemm_tc", "bound": "tensor", "achieved": ach, "peak": peak,
                         "unit": "TOP/s", "frac": ach / peak,
-                        "traffic": NCU_TRAFFIC_CFG3.get("k_gemm_tc") if wl.name == "cfg3" else None,
+                        "traffic": traffic_of("k_gemm_tc"),
                         "peak_note": f"int8 = 2 x {peaks['source']} bf16 burst peak"}
         else:
             n = names[dom]
             ach = alg[n] / (us[dom] * 1e-6) / 1e9
             roofline = {"kernel": kernel_names[n], "bound": "hbm", "achieved": ach,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
-                        "traffic": NCU_TRAFFIC_CFG3.get(kernel_names[n]) if wl.name == "cfg3" else None,
+                        "traffic": traffic_of(kernel_names[n]),
                         "peak_note": f"of {peaks['source']}"}
     # measured int8 tensor rate of this device: an MMA-only probe kernel (operands in
     # shared memory, accumulators in tensor memory), timed with CUDA events
@@ -366,6 +463,75 @@ def run_ours(args, wl):
                   "roofline_us": max(t_mma, t_hbm) * 1e6,
                   "frac": max(t_mma, t_hbm) / (ms_local / args.steps * 1e-3),
                   "peaks": peaks["source"]}
+    # third term, which the two-term definition leaves out: plain instruction issue.  Warp
+    # instructions per step (ncu smsp__inst_executed.sum, profiles/traffic.json) over
+    # SMs x 4 schedulers x 1 instruction per cycle at the maximum SM clock.
+    if wl.name == "cfg3" and not single_kernel:
+        cnt = load_counters()
+        inst = [(cnt.get(k) or {}).get("inst_executed") for k in kernel_names.values()]
+        if all(v is not None for v in inst):
+            sms = torch.cuda.get_device_properties(dev).multi_processor_count
+            t_issue = sum(inst) / (sms * 4 * 1.965e9)
+            layer_roof["three_term"] = {
+                "warp_instructions_per_step": int(sum(inst)), "t_issue_us": t_issue * 1e6,
+                "roofline_us": max(t_mma, t_hbm, t_issue) * 1e6,
+                "frac": max(t_mma, t_hbm, t_issue) / (ms_local / args.steps * 1e-3)}
+
+    # ---- the same steps with every buffer resident in L2 (one buffer set): warm-L2 figure ----
+    wg_ = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(wg_, stream=side):
+            for i in range(chunk):
+                plan.conv_forward(xs[0], Us[0], b_dev, ys[0], ws)
+    torch.cuda.synchronize()
+    wg_.replay()
+    torch.cuda.synchronize()
+    w0, w1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    w0.record()
+    for _ in range(10):
+        wg_.replay()
+    w1.record()
+    torch.cuda.synchronize()
+    warm_us = w0.elapsed_time(w1) * 1e3 / (10 * chunk)
+    # restore the workspace contents of a complete rotating step
+    step(0)
+    torch.cuda.synchronize()
+
+    # ---- the single-launch layer kernel on the same workload (extra, not the headline
+    #      unless the plan chose it) ----
+    single_launch = None
+    if rank == 0 and plan.path != binding.PATH_FUSED_LAYER:
+        try:
+            plan_f = make_plan(s_V, s_U, s_M, s_Y, path=binding.PATH_FUSED_LAYER)
+        except binding.WinoError:
+            plan_f = None
+        if plan_f is not None:
+            def fstep(i):
+                j = i % R
+                plan_f.conv_forward(xs[j], Us[j], b_dev, ys[j], ws)
+            for i in range(3):
+                fstep(i)
+            torch.cuda.synchronize()
+            fg = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(fg, stream=side):
+                    for i in range(chunk):
+                        fstep(i)
+            torch.cuda.synchronize()
+            fg.replay()
+            torch.cuda.synchronize()
+            f0_, f1_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            f0_.record()
+            for _ in range(10):
+                fg.replay()
+            f1_.record()
+            torch.cuda.synchronize()
+            fus = f0_.elapsed_time(f1_) * 1e3 / (10 * chunk)
+            single_launch = {"kernel": "k_layer_fused", "us": fus, "launches_per_step": 1,
+                             "value": direct_ops(wl, wl.N) / (fus * 1e-6) / 1e12, "unit": UNIT,
+                             "frac": max(t_mma, t_hbm) * 1e6 / fus, "status": plan_f.last_status()}
+            step(0)
+            torch.cuda.synchronize()
 
     # ---- extra, not the headline: two independent steps in flight on two streams
     #      (each with its own plan and workspace), as a serving loop would run them ----
@@ -489,6 +655,28 @@ def run_ours(args, wl):
                                   dist if world > 1 else None)
     clocks = sampler.stop() if rank == 0 else None
 
+    # ---- the other configurations (timing only; parity is the GPU tests' job) ----
+    other = None
+    if rank == 0 and world == 1 and not args.no_other_configs:
+        other = []
+        for name in ("cfg2", "cfg4"):
+            if name == wl.name:
+                continue
+            o = wi.CONFIGS[name]
+            us, pth = time_layer_quick(binding, cook_toom, torch, dev, o.N, o.C, o.H, o.W, o.K, o.m,
+                                       flex_seed=o.seed if o.flex else None)
+            if us is not None:
+                other.append(layer_row(peaks, name, o.N, o.C, o.H, o.W, o.K, o.m, us, pth))
+        for ly in wi.resnet18_layers(1005, 256):
+            if ly["m"] == 0:
+                continue      # stride-2 layers are direct convolutions, not timed
+            us, pth = time_layer_quick(binding, cook_toom, torch, dev, ly["N"], ly["C"], ly["H"],
+                                       ly["W"], ly["K"], ly["m"])
+            if us is not None:
+                other.append(layer_row(peaks, f"cfg5.conv{ly['index']}", ly["N"], ly["C"], ly["H"],
+                                       ly["W"], ly["K"], ly["m"], us, pth))
+        torch.cuda.empty_cache()
+
     # ---- the oracle beside it (rank 0, single GPU runs only) ----
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -518,9 +706,13 @@ def run_ours(args, wl):
             "config": workload_config(
                 wl, f"inputs rotate over {R} buffer sets ({R * (xb + yb + plan.weight_bytes) / 1e6:.0f} MB > L2)"),
             "wino_domain_TOPS": wino_ops(wl, wl.N) * world / (ms_per_step * 1e-3) / 1e12,
-            "path": {1: "staged_tc", 2: "staged_dp4a", 3: "smallc", 4: "staged_tc_ptr", 5: "fused_f2"}[plan.path],
+            "path": PATH_NAMES[plan.path],
             "gpu_launches": launches_per_step * args.steps,
             "roofline": roofline, "layer_roofline": layer_roof, "stages": stages,
+            "warm_l2": {"ms_per_step": warm_us * 1e-3,
+                        "value": direct_ops(wl, wl.N) / (warm_us * 1e-6) / 1e12, "unit": UNIT,
+                        "note": "every step on one buffer set (x, U_q, y stay in L2)"},
+            "single_launch": single_launch, "other_configs": other,
             "int8_mma_probe_TOPS": mma_probe,
             "weight_transform": {"us": wt_us, "GBps": wt_bytes / (wt_us * 1e-6) / 1e9,
                                  "algorithmic_bytes": wt_bytes},
@@ -542,6 +734,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg3", choices=sorted(wi.CONFIGS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-other-configs", action="store_true",
+                    help="skip the timing rows of cfg2, cfg4 and the cfg5 layers")
+    ap.add_argument("--path", type=int, default=0,
+                    help="pin the execution path (WINO_PATH_* number; 0 = the plan's own choice)")
     args = ap.parse_args()
     wl = wi.CONFIGS[args.workload]
     if args.impl == "reference":

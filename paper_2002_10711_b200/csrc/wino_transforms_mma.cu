@@ -175,13 +175,13 @@ k_input_transform_mma(const __grid_constant__ Params p, const __grid_constant__ 
         // refill the slot of unit i-1 once its MMAs have read it
         if (i >= 1 && i - 1 + kInSlots < n_my) {
           const uint32_t sl = (uint32_t)((i - 1) % kInSlots);
-          if (!mbar_wait(s.bar_in_empty + 8u * sl, (uint32_t)((i - 1) / kInSlots) & 1u, abort_p)) { ok = false; break; }
+          if (!mbar_wait<false>(s.bar_in_empty + 8u * sl, (uint32_t)((i - 1) / kInSlots) & 1u, abort_p)) { ok = false; break; }
           issue(i - 1 + kInSlots);
         }
         const uint32_t sl = (uint32_t)(i % kInSlots);
-        if (!mbar_wait(s.bar_full + 8u * sl, (uint32_t)(i / kInSlots) & 1u, abort_p)) { ok = false; break; }
+        if (!mbar_wait<false>(s.bar_full + 8u * sl, (uint32_t)(i / kInSlots) & 1u, abort_p)) { ok = false; break; }
         const int b = i & 1;
-        if (!mbar_wait(s.bar_acc_empty + 8u * b, ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_p)) { ok = false; break; }
+        if (!mbar_wait<false>(s.bar_acc_empty + 8u * b, ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_p)) { ok = false; break; }
         tc_fence_after();
         const uint64_t da = desc_mnmajor_sw128(s.in + sl * L::kInSlot);
 #pragma unroll
@@ -203,7 +203,7 @@ k_input_transform_mma(const __grid_constant__ Params p, const __grid_constant__ 
       const int tau = u / cchunks, c0 = (u - tau * cchunks) << 7;
       const int b = i & 1;
       if (et == 0) {
-        if (!mbar_wait(s.bar_acc_full + 8u * b, (uint32_t)(i >> 1) & 1u, abort_p)) *abort_p = 1u;
+        if (!mbar_wait<false>(s.bar_acc_full + 8u * b, (uint32_t)(i >> 1) & 1u, abort_p)) *abort_p = 1u;
         bulk_wait_read_n<1>();                  // the store that last read staging tile b is done
       }
       epi_barrier();
@@ -232,12 +232,13 @@ k_input_transform_mma(const __grid_constant__ Params p, const __grid_constant__ 
       __syncwarp();
       if (lane == 0) mbar_arrive(s.bar_acc_empty + 8u * b);
       const uint32_t wr = s.out + (uint32_t)b * L::kOut + (uint32_t)c;
+      // all codes first (independent chains the compiler can interleave), then the stores
 #pragma unroll
-      for (int xi = 0; xi < T2; ++xi) {
-        const float r = fminf(fmaxf(__fmaf_rn(__int2float_rn((int)v[xi]), p.mult_V, kMagic), lo), hi);
-        asm volatile("st.shared.u8 [%0], %1;" ::"r"(wr + (uint32_t)xi * 128u), "r"(__float_as_uint(r))
-                     : "memory");
-      }
+      for (int xi = 0; xi < T2; ++xi)
+        v[xi] = __float_as_uint(fminf(fmaxf(__fmaf_rn(__int2float_rn((int)v[xi]), p.mult_V, kMagic), lo), hi));
+      uint8_t* sp = gen + (wr - base);
+#pragma unroll
+      for (int xi = 0; xi < T2; ++xi) sp[xi * 128] = (uint8_t)v[xi];
       fence_async_smem();
       epi_barrier();
       if (et == 0) {
@@ -328,13 +329,13 @@ k_output_transform_mma(const __grid_constant__ Params p, const __grid_constant__
       for (int i = 0; i < n_my; ++i) {
         if (i >= 1 && i - 1 + kInSlots < n_my) {
           const uint32_t sl = (uint32_t)((i - 1) % kInSlots);
-          if (!mbar_wait(s.bar_in_empty + 8u * sl, (uint32_t)((i - 1) / kInSlots) & 1u, abort_p)) { ok = false; break; }
+          if (!mbar_wait<false>(s.bar_in_empty + 8u * sl, (uint32_t)((i - 1) / kInSlots) & 1u, abort_p)) { ok = false; break; }
           issue(i - 1 + kInSlots);
         }
         const uint32_t sl = (uint32_t)(i % kInSlots);
-        if (!mbar_wait(s.bar_full + 8u * sl, (uint32_t)(i / kInSlots) & 1u, abort_p)) { ok = false; break; }
+        if (!mbar_wait<false>(s.bar_full + 8u * sl, (uint32_t)(i / kInSlots) & 1u, abort_p)) { ok = false; break; }
         const int b = i & 1;
-        if (!mbar_wait(s.bar_acc_empty + 8u * b, ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_p)) { ok = false; break; }
+        if (!mbar_wait<false>(s.bar_acc_empty + 8u * b, ((uint32_t)(i >> 1) & 1u) ^ 1u, abort_p)) { ok = false; break; }
         tc_fence_after();
         const uint64_t da = desc_mnmajor_sw128(s.in + sl * L::kInSlot);
 #pragma unroll
@@ -356,7 +357,7 @@ k_output_transform_mma(const __grid_constant__ Params p, const __grid_constant__
       const int tau = t0 + i * tstride;
       const int b = i & 1;
       if (et == 0) {
-        if (!mbar_wait(s.bar_acc_full + 8u * b, (uint32_t)(i >> 1) & 1u, abort_p)) *abort_p = 1u;
+        if (!mbar_wait<false>(s.bar_acc_full + 8u * b, (uint32_t)(i >> 1) & 1u, abort_p)) *abort_p = 1u;
         bulk_wait_read_n<1>();
       }
       epi_barrier();
@@ -375,9 +376,11 @@ k_output_transform_mma(const __grid_constant__ Params p, const __grid_constant__
       for (int q = 0; q < MM; ++q) {
         const float yf = __fmaf_rn(__int2float_rn((int)v[q]), p.mult_Y, b_scaled);
         const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
-        const uint32_t code = (uint32_t)(magic_to_int(r) + p.z_Y);
-        asm volatile("st.shared.u8 [%0], %1;" ::"r"(wr + (uint32_t)q * 128u), "r"(code) : "memory");
+        v[q] = (uint32_t)(magic_to_int(r) + p.z_Y);
       }
+      uint8_t* sp = gen + (wr - base);
+#pragma unroll
+      for (int q = 0; q < MM; ++q) sp[q * 128] = (uint8_t)v[q];
       fence_async_smem();
       epi_barrier();
       if (et == 0) {
