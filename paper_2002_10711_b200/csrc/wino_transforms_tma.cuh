@@ -70,6 +70,13 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   if (threadIdx.x == 0) {
     tma_prefetch_map(&mapX);
     tma_prefetch_map(&mapV);
+    // ask for the patches to be brought into L2 while the preceding kernel is still running
+    // (a hint only: nothing is read into the SM before the wait below)
+    for (int i = 0; i < ntile; ++i) {
+      const int tau = tau0 + i;
+      tma_prefetch_l2_4d(&mapX, c0, (tau % p.TW) * M - 1, ((tau / p.TW) % p.TH) * M - 1,
+                         tau / (p.TW * p.TH));
+    }
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
     mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
     for (int i = 0; i < ntile; ++i) {
