@@ -216,6 +216,14 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
   if (warp == 0 && lane == 0) {   // descriptors do not depend on the previous kernel
     tma_prefetch_map(&mapV);
     tma_prefetch_map(&mapU);
+    // nor do the transformed weights: ask for the U_q tiles of this CTA's first two items to
+    // be brought into L2 while the preceding kernel is still running (a hint only)
+    int n = 0;
+    for (int it = blockIdx.x; it < a.n_items && n < 2; it += gridDim.x, ++n) {
+      const int xi = it / per_xi, rem = it - xi * per_xi;
+      const int nb = rem / a.n_mblk;
+      for (int kb = 0; kb < KB; ++kb) tma_prefetch_l2_3d(&mapU, kb * kStageK, nb * a.BN, xi);
+    }
   }
   tc_fence_before();
   __syncthreads();

@@ -271,12 +271,11 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
       tma_prefetch_map(&mapX);
       tma_prefetch_map(&mapMld);
     }
-    griddep_wait();
-    if (lane == 0) WINO_TRACE_AT(1);
-    if (lane >= kSlots) {
-      // x comes from HBM: the idle lanes ask for the patches of the units beyond the first
-      // round to be brought into L2 now, so that the loads below find them there
-      for (int jj = lane; jj < nA && jj < kPrefetchUnits; jj += 32 - kSlots) {
+    {
+      // x comes from HBM: ask for the patches of this CTA's units to be brought into L2 while
+      // the preceding kernel is still running (a hint only: nothing reaches the SM before the
+      // wait below), so that the loads find them there
+      for (int jj = lane; jj < nA && jj < kPrefetchUnits; jj += 32) {
         const int u = cta + jj * grid;
         const int tau = u / cchunks, c0 = (u - tau * cchunks) << 7;
         const int tw = tau % p.TW;
@@ -284,7 +283,10 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
         const int n = tau / (p.TW * p.TH);
         tma_prefetch_l2_4d(&mapX, c0, tw * M - 1, th * M - 1, n);
       }
-    } else {
+    }
+    griddep_wait();
+    if (lane == 0) WINO_TRACE_AT(1);
+    if (lane < kSlots) {
       const uint32_t sl = (uint32_t)lane;
       int jj = lane, it = 0;
       const long long t0 = clock64();
