@@ -13,6 +13,18 @@ equivalent int8 TOPS: 2*N*H*W*K*C*9 operations per step over the measured time.
 Prints ONE JSON line (rank 0).  With torchrun (N > 1) every rank processes its
 own batch (weak scaling, no collective on the data path); time is the max over
 ranks, value the sum of work over that time.
+
+Beside the contract's keys the line carries: `stages` (each kernel of a step
+timed alone), `roofline` (the dominant kernel; `traffic` = its DRAM bytes per
+launch from profiles/traffic.json while the digest stored there matches the CUDA
+sources, else null), `layer_roofline` (whole step against max(t_MMA, t_HBM), and
+`three_term` with the ALU issue bound from the same counters), `warm_l2` (every
+step on one buffer set), `single_launch` (the one-kernel layer path on the same
+workload), `other_configs` (cfg2, cfg4 and the Winograd layers of the ResNet-18
+body, one row each), `overlapped_steps`, `int8_mma_probe_TOPS`,
+`weight_transform`, `e2e`, `cpu_baseline`, `clocks`.  `--path P` forces a path of
+the library, `--no-other-configs` and `--no-cpu-baseline` shorten the run (used
+for profiler captures).
 """
 from __future__ import annotations
 
