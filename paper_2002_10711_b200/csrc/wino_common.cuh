@@ -41,6 +41,36 @@ __device__ __forceinline__ float quant_magic(float v, float mult, float lo, floa
   return fminf(fmaxf(r, __fadd_rn(lo, kMagic)), __fadd_rn(hi, kMagic));
 }
 __device__ __forceinline__ int magic_to_int(float r) { return __float_as_int(r) - kMagicBits; }
+
+// Saturating pack of two 32-bit integers to signed bytes (cvt.pack.sat): byte 1 = sat(a),
+// byte 0 = sat(b), upper half = lower half of c.
+__device__ __forceinline__ uint32_t pack_sat_s8(int a, int b, uint32_t c) {
+  uint32_t d;
+  asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
+}
+
+// Four codes of one row as a little-endian packed word.  HI127: the upper bound of the
+// quantizer is +127 and is applied by the saturating pack (which also covers products too
+// large for the rounding constant: their bit patterns stay above it); the lower bound, any
+// code >= -128, is applied on the float.  Otherwise both bounds are applied on the float.
+template <bool HI127>
+__device__ __forceinline__ uint32_t quant_pack4(float v0, float v1, float v2, float v3, float mult,
+                                                float lo_magic, float hi_magic) {
+  if constexpr (HI127) {
+    const int c0 = magic_to_int(fmaxf(__fmaf_rn(v0, mult, kMagic), lo_magic));
+    const int c1 = magic_to_int(fmaxf(__fmaf_rn(v1, mult, kMagic), lo_magic));
+    const int c2 = magic_to_int(fmaxf(__fmaf_rn(v2, mult, kMagic), lo_magic));
+    const int c3 = magic_to_int(fmaxf(__fmaf_rn(v3, mult, kMagic), lo_magic));
+    return pack_sat_s8(c1, c0, pack_sat_s8(c3, c2, 0u));
+  } else {
+    const uint32_t r0 = __float_as_uint(fminf(fmaxf(__fmaf_rn(v0, mult, kMagic), lo_magic), hi_magic));
+    const uint32_t r1 = __float_as_uint(fminf(fmaxf(__fmaf_rn(v1, mult, kMagic), lo_magic), hi_magic));
+    const uint32_t r2 = __float_as_uint(fminf(fmaxf(__fmaf_rn(v2, mult, kMagic), lo_magic), hi_magic));
+    const uint32_t r3 = __float_as_uint(fminf(fmaxf(__fmaf_rn(v3, mult, kMagic), lo_magic), hi_magic));
+    return __byte_perm(__byte_perm(r0, r1, 0x0040u), __byte_perm(r2, r3, 0x0040u), 0x5410u);
+  }
+}
 __device__ __forceinline__ float magic_to_float(float r) { return __fsub_rn(r, kMagic); }
 
 // int8 byte `sel` (0..3) of a packed word, minus zero point z, as an exact float:

@@ -115,15 +115,19 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
         dst[q] = make_int4((int)r[4 * q], (int)r[4 * q + 1], (int)r[4 * q + 2], (int)r[4 * q + 3]);
   } else {
     uint32_t w[8];
+    const float lo_m = __fadd_rn(p.lo_M, kMagic), hi_m = __fadd_rn(p.hi_M, kMagic);
+    if (p.hi_M == 127.0f) {
 #pragma unroll
-    for (int q = 0; q < 8; ++q) {
-      const float f0 = quant_magic(acc_to_float<SMALL>(r[4 * q + 0]), p.mult_M, p.lo_M, p.hi_M);
-      const float f1 = quant_magic(acc_to_float<SMALL>(r[4 * q + 1]), p.mult_M, p.lo_M, p.hi_M);
-      const float f2 = quant_magic(acc_to_float<SMALL>(r[4 * q + 2]), p.mult_M, p.lo_M, p.hi_M);
-      const float f3 = quant_magic(acc_to_float<SMALL>(r[4 * q + 3]), p.mult_M, p.lo_M, p.hi_M);
-      const uint32_t lo = __byte_perm(__float_as_uint(f0), __float_as_uint(f1), 0x0040u);
-      const uint32_t hi = __byte_perm(__float_as_uint(f2), __float_as_uint(f3), 0x0040u);
-      w[q] = __byte_perm(lo, hi, 0x5410u);
+      for (int q = 0; q < 8; ++q)
+        w[q] = quant_pack4<true>(acc_to_float<SMALL>(r[4 * q + 0]), acc_to_float<SMALL>(r[4 * q + 1]),
+                                 acc_to_float<SMALL>(r[4 * q + 2]), acc_to_float<SMALL>(r[4 * q + 3]),
+                                 p.mult_M, lo_m, hi_m);
+    } else {
+#pragma unroll
+      for (int q = 0; q < 8; ++q)
+        w[q] = quant_pack4<false>(acc_to_float<SMALL>(r[4 * q + 0]), acc_to_float<SMALL>(r[4 * q + 1]),
+                                  acc_to_float<SMALL>(r[4 * q + 2]), acc_to_float<SMALL>(r[4 * q + 3]),
+                                  p.mult_M, lo_m, hi_m);
     }
     uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(out) + o);
     if (FULL || k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);

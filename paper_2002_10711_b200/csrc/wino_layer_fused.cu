@@ -640,15 +640,18 @@ k_layer_fused(const __grid_constant__ Params p, const __grid_constant__ CUtensor
           const int k0 = nb * a.BN + col;
           if (tau < p.T && k0 < p.K) {
             uint32_t w[8];
+            if (p.hi_M == 127.0f) {
 #pragma unroll
-            for (int q = 0; q < 8; ++q) {
-              float f[4];
+              for (int q = 0; q < 8; ++q)
+                w[q] = quant_pack4<true>(__int2float_rn((int)r[4 * q]), __int2float_rn((int)r[4 * q + 1]),
+                                         __int2float_rn((int)r[4 * q + 2]), __int2float_rn((int)r[4 * q + 3]),
+                                         p.mult_M, lo, hi);
+            } else {
 #pragma unroll
-              for (int e = 0; e < 4; ++e)
-                f[e] = fminf(fmaxf(__fmaf_rn(__int2float_rn((int)r[4 * q + e]), p.mult_M, kMagic), lo), hi);
-              const uint32_t l2 = __byte_perm(__float_as_uint(f[0]), __float_as_uint(f[1]), 0x0040u);
-              const uint32_t h2 = __byte_perm(__float_as_uint(f[2]), __float_as_uint(f[3]), 0x0040u);
-              w[q] = __byte_perm(l2, h2, 0x5410u);
+              for (int q = 0; q < 8; ++q)
+                w[q] = quant_pack4<false>(__int2float_rn((int)r[4 * q]), __int2float_rn((int)r[4 * q + 1]),
+                                          __int2float_rn((int)r[4 * q + 2]), __int2float_rn((int)r[4 * q + 3]),
+                                          p.mult_M, lo, hi);
             }
             uint4* dst = reinterpret_cast<uint4*>(mq + ((long)xi * p.T + tau) * p.K + k0);
             dst[0] = make_uint4(w[0], w[1], w[2], w[3]);

@@ -130,7 +130,7 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   if (threadIdx.x == 0) {
     tma_store_3d(&mapV, s_out, c0, tau0, 0);
     bulk_commit();
-    bulk_wait_read();   // shared memory may be released; the grid's completion publishes the data
+    bulk_wait_all();    // the bytes are in place before the block leaves
   }
 }
 
@@ -236,7 +236,7 @@ k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_const
   }
   // shared memory may be released once the stores have read it; the grid's completion
   // publishes the data
-  if (threadIdx.x == 0) bulk_wait_read();
+  if (threadIdx.x == 0) bulk_wait_all();
 }
 
 template <int M, int MODE, int KC, int G, int CPT>
@@ -329,7 +329,7 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
       tma_store_4d(&mapY, s_out + (uint32_t)i * kTileOut, k0, tw * M, th * M, n);
     }
     bulk_commit();
-    bulk_wait_read();
+    bulk_wait_all();
   }
 }
 
