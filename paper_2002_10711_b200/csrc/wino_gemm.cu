@@ -12,6 +12,7 @@
 //                 ALUs; fallback for channel counts the TMA path cannot take.
 #include "wino_launch.h"
 #include "wino_ptx.cuh"
+#include "wino_trace.cuh"
 
 namespace wino {
 
@@ -78,6 +79,11 @@ int launch_gemm_dp4a(const Params& p, const LaunchOpt& o, const int8_t* Vq, cons
 // consumes 32 channels.
 // ---------------------------------------------------------------------------
 
+#ifdef WINO_TRACE
+static __device__ TraceTable g_gemm_trace;
+#endif
+WINO_ST_READER(wino_trace_gemm, g_gemm_trace)
+
 constexpr int kEpiWarps = 16;
 constexpr int kGemmThreads = 64 + 32 * kEpiWarps;
 
@@ -130,8 +136,15 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
                                   p.mult_M, lo_m, hi_m);
     }
     uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(out) + o);
-    if (FULL || k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-    if (FULL || k0 + 16 < p.K) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    if constexpr (FULL) {
+      // the whole 32-byte sector of this row in one request
+      asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]),
+                   "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                   : "memory");
+    } else {
+      if (k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      if (k0 + 16 < p.K) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+    }
   }
 }
 
@@ -140,7 +153,9 @@ template <bool SMALL, bool FULL, bool STATS>
 __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs& a, void* out,
                                               unsigned* absmaxM, uint32_t tmem_base,
                                               uint32_t bar_acc_full, uint32_t bar_acc_empty,
-                                              volatile uint32_t* abort_p, int warp, int lane) {
+                                              volatile uint32_t* abort_p, int warp, int lane,
+                                              int trace_step) {
+  (void)trace_step;
   const int quad = warp & 3;
   const int sub = (warp - 2) >> 2;
   const int per_xi = a.n_mblk * a.n_nblk;
@@ -155,6 +170,7 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
       *abort_p = 1u;
       break;
     }
+    if (warp == 2 && lane == 0 && li < 2) WINO_ST(g_gemm_trace, trace_step, 5 + 2 * li);
     tc_fence_after();
     const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride) + ((uint32_t)(quad * 32) << 16);
     // the accumulator holds MB blocks of BN columns side by side; one chunk at a
@@ -175,6 +191,7 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
     tc_fence_before();
     __syncwarp();
     if (lane == 0) mbar_arrive(bar_acc_empty + 8u * buf);
+    if (warp == 2 && lane == 0 && li < 2) WINO_ST(g_gemm_trace, trace_step, 6 + 2 * li);
   }
   if constexpr (STATS) atomic_absmax(absmaxM, vmax);
 }
@@ -203,6 +220,14 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
   const int KB = (p.C + kStageK - 1) / kStageK;
   const int per_xi = a.n_mblk * a.n_nblk;
 
+  int trace_step = 0;
+#ifdef WINO_TRACE
+  int& trace_step_s = *reinterpret_cast<int*>(gen + (abort_slot + 4u - base));
+  if (threadIdx.x == 0) {
+    WINO_ST_BEGIN(g_gemm_trace, trace_step_s);
+    WINO_ST(g_gemm_trace, trace_step_s, 0);
+  }
+#endif
   griddep_launch();
   if (threadIdx.x == 0) {
     for (int s = 0; s < a.stages; ++s) {
@@ -233,7 +258,12 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot_p;
+#ifdef WINO_TRACE
+  trace_step = trace_step_s;
+  if (threadIdx.x == 0) WINO_ST(g_gemm_trace, trace_step, 1);
+#endif
   griddep_wait();   // everything below reads or writes buffers other kernels touch
+  if (threadIdx.x == 0) WINO_ST(g_gemm_trace, trace_step, 2);
 
   if (warp == 0) {
     if (lane == 0) {
@@ -269,6 +299,10 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
         const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride);
         for (int kb = 0; kb < KB && ok; ++kb) {
           if (!mbar_wait(bar_full + 8u * s, ph, abort_p)) { ok = false; break; }
+          if (li == 0 && kb == 0) WINO_ST(g_gemm_trace, trace_step, 3);
+          if (li == 0 && kb == KB - 1) WINO_ST(g_gemm_trace, trace_step, 4);
+          if (li == 1 && kb == 0) WINO_ST(g_gemm_trace, trace_step, 10);
+          if (li == 1 && kb == KB - 1) WINO_ST(g_gemm_trace, trace_step, 11);
           tc_fence_after();
           const uint32_t sa = base + (uint32_t)s * stage_bytes;
           const uint64_t db = make_desc_sw128(sa + (uint32_t)a.MB * a_bytes);
@@ -294,21 +328,22 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     const bool full = (p.K % a.BN) == 0 && (a.BN % 32) == 0;
     if (absmaxM != nullptr)
       epilogue_loop<false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
-                                        abort_p, warp, lane);
+                                        abort_p, warp, lane, trace_step);
     else if (small && full)
       epilogue_loop<true, true, false>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
-                                       abort_p, warp, lane);
+                                       abort_p, warp, lane, trace_step);
     else if (full)
       epilogue_loop<false, true, false>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
-                                        abort_p, warp, lane);
+                                        abort_p, warp, lane, trace_step);
     else
       epilogue_loop<false, false, false>(p, a, out, absmaxM, tmem_base, bar_acc_full,
-                                         bar_acc_empty, abort_p, warp, lane);
+                                         bar_acc_empty, abort_p, warp, lane, trace_step);
   }
   __syncwarp();
   tc_fence_before();
   __syncthreads();
   if (*abort_p != 0u && threadIdx.x == 0) atomicExch(status, -6);  // WINO_ERR_TIMEOUT
+  if (threadIdx.x == 0) WINO_ST(g_gemm_trace, trace_step, 9);
   if (warp == 1) {
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);

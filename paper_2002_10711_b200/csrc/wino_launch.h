@@ -2,6 +2,7 @@
 // translation units.  Every function enqueues work on `st` and returns 0 or a
 // negative WINO_ERR_* code; none allocates or synchronizes.
 #pragma once
+#include <cstdio>
 #include <mutex>
 
 #include <cuda.h>
@@ -44,8 +45,13 @@ class DeviceOnce {
 template <typename Kern>
 int set_max_smem(DeviceOnce& once, int dev, Kern kernel, size_t smem) {
   return once.run(dev, [&]() -> int {
-    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) ==
-                   cudaSuccess ? 0 : -5;
+    const cudaError_t e =
+        cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+#ifdef WINO_TRACE
+    if (e != cudaSuccess)
+      std::fprintf(stderr, "shared-memory attribute failed: %s (%zu bytes)\n", cudaGetErrorString(e), smem);
+#endif
+    return e == cudaSuccess ? 0 : -5;
   });
 }
 
@@ -145,7 +151,13 @@ int launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, 
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = pdl ? 1 : 0;
-  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...) == cudaSuccess ? 0 : -5;
+  const cudaError_t e = cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+#ifdef WINO_TRACE
+  if (e != cudaSuccess)
+    std::fprintf(stderr, "launch failed: %s (grid %u block %u smem %zu)\n", cudaGetErrorString(e), grid.x,
+                 block.x, smem);
+#endif
+  return e == cudaSuccess ? 0 : -5;
 }
 
 }  // namespace wino

@@ -12,6 +12,7 @@
 // address arithmetic, which was a third of their instructions.
 #pragma once
 #include "wino_ptx.cuh"
+#include "wino_trace.cuh"
 
 namespace wino {
 
@@ -38,6 +39,14 @@ __device__ __forceinline__ void sts_pack(uint32_t addr, uint32_t v) {
   }
 }
 
+#ifdef WINO_TRACE
+static __device__ TraceTable g_in_trace, g_out_trace;
+#endif
+#if WINO_M == 4
+WINO_ST_READER(wino_trace_input, g_in_trace)
+WINO_ST_READER(wino_trace_output, g_out_trace)
+#endif
+
 template <int M, int MODE, int CC, int G, int CPT>
 __global__ void __launch_bounds__((CC / CPT) * G)
 k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
@@ -60,6 +69,12 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   const int g = threadIdx.x / TPT, c4 = threadIdx.x % TPT;
   const int ntile = min(G, p.T - tau0);
 
+  int trace_step = 0;
+  (void)trace_step;
+  if (threadIdx.x == 0) {
+    WINO_ST_BEGIN(g_in_trace, trace_step);
+    WINO_ST(g_in_trace, trace_step, 0);
+  }
   griddep_launch();
   if (threadIdx.x == 0) {
     mbar_init(bar, 1);
@@ -78,6 +93,7 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
                          tau / (p.TW * p.TH));
     }
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
+    WINO_ST(g_in_trace, trace_step, 1);
     mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
     for (int i = 0; i < ntile; ++i) {
       const int tau = tau0 + i;
@@ -91,6 +107,7 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
       abort_flag = 1u;
       atomicExch(status, -6);  // WINO_ERR_TIMEOUT
     }
+    WINO_ST(g_in_trace, trace_step, 2);
   }
   __syncthreads();
   if (*(volatile uint32_t*)&abort_flag != 0u) return;
@@ -128,9 +145,11 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   fence_async_smem();
   __syncthreads();
   if (threadIdx.x == 0) {
+    WINO_ST(g_in_trace, trace_step, 3);
     tma_store_3d(&mapV, s_out, c0, tau0, 0);
     bulk_commit();
     bulk_wait_all();    // the bytes are in place before the block leaves
+    WINO_ST(g_in_trace, trace_step, 4);
   }
 }
 
@@ -262,6 +281,12 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
   const int g = threadIdx.x / TPT, k4 = threadIdx.x % TPT;
   const int ntile = min(G, p.T - tau0);
 
+  int trace_step = 0;
+  (void)trace_step;
+  if (threadIdx.x == 0) {
+    WINO_ST_BEGIN(g_out_trace, trace_step);
+    WINO_ST(g_out_trace, trace_step, 0);
+  }
   griddep_launch();
   if (threadIdx.x == 0) {
     mbar_init(bar, 1);
@@ -273,12 +298,14 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     tma_prefetch_map(&mapM);
     tma_prefetch_map(&mapY);
     griddep_wait();
+    WINO_ST(g_out_trace, trace_step, 1);
     mbar_expect_tx(bar, kInBytes);   // the full box counts, clipped rows included
     tma_load_3d(s_in, &mapM, bar, k0, tau0, 0);
     if (!mbar_wait(bar, 0u, &abort_flag)) {
       abort_flag = 1u;
       atomicExch(status, -6);  // WINO_ERR_TIMEOUT
     }
+    WINO_ST(g_out_trace, trace_step, 2);
   }
   __syncthreads();
   if (*(volatile uint32_t*)&abort_flag != 0u) return;
@@ -321,6 +348,7 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
   fence_async_smem();
   __syncthreads();
   if (threadIdx.x == 0) {
+    WINO_ST(g_out_trace, trace_step, 3);
     for (int i = 0; i < ntile; ++i) {
       const int tau = tau0 + i;
       const int tw = tau % p.TW;
@@ -330,6 +358,7 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     }
     bulk_commit();
     bulk_wait_all();
+    WINO_ST(g_out_trace, trace_step, 4);
   }
 }
 
