@@ -240,19 +240,25 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     }
     *abort_p = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+#ifdef WINO_TRACE
+    WINO_ST(g_gemm_trace, trace_step_s, 12);
+#endif
   }
-  if (warp == 1) tmem_alloc(tmem_slot, (uint32_t)a.tmem_cols);
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, (uint32_t)a.tmem_cols);
+#ifdef WINO_TRACE
+    if (lane == 0) *reinterpret_cast<unsigned long long*>(gen + (tmem_slot + 16u - base)) = trace_now();
+#endif
+  }
   if (warp == 0 && lane == 0) {   // descriptors do not depend on the previous kernel
     tma_prefetch_map(&mapV);
     tma_prefetch_map(&mapU);
-    // nor do the transformed weights: ask for the U_q tiles of this CTA's first two items to
-    // be brought into L2 while the preceding kernel is still running (a hint only)
-    int n = 0;
-    for (int it = blockIdx.x; it < a.n_items && n < 2; it += gridDim.x, ++n) {
-      const int xi = it / per_xi, rem = it - xi * per_xi;
-      const int nb = rem / a.n_mblk;
-      for (int kb = 0; kb < KB; ++kb) tma_prefetch_l2_3d(&mapU, kb * kStageK, nb * a.BN, xi);
-    }
+#ifdef WINO_TRACE
+    WINO_ST(g_gemm_trace, trace_step_s, 14);
+#endif
+#ifdef WINO_TRACE
+    WINO_ST(g_gemm_trace, trace_step_s, 15);
+#endif
   }
   tc_fence_before();
   __syncthreads();
@@ -260,7 +266,10 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
   const uint32_t tmem_base = *tmem_slot_p;
 #ifdef WINO_TRACE
   trace_step = trace_step_s;
-  if (threadIdx.x == 0) WINO_ST(g_gemm_trace, trace_step, 1);
+  if (threadIdx.x == 0) {
+    WINO_ST(g_gemm_trace, trace_step, 1);
+    g_gemm_trace.t[trace_step][blockIdx.x][13] = *reinterpret_cast<unsigned long long*>(gen + (tmem_slot + 16u - base));
+  }
 #endif
   griddep_wait();   // everything below reads or writes buffers other kernels touch
   if (threadIdx.x == 0) WINO_ST(g_gemm_trace, trace_step, 2);
@@ -308,11 +317,19 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
           const uint64_t db = make_desc_sw128(sa + (uint32_t)a.MB * a_bytes);
           const int remc = p.C - kb * kStageK;
           const int ksteps = remc >= kStageK ? 4 : (remc + 31) / 32;
+          // (few instructions per MMA: this thread shares its scheduler with epilogue warps)
           for (int j = 0; j < a.MB; ++j) {
             const uint64_t da = make_desc_sw128(sa + (uint32_t)j * a_bytes);
-            for (int k = 0; k < ksteps; ++k)
-              mma_i8(tacc + (uint32_t)(j * a.BN), da + (uint64_t)(k * 2), db + (uint64_t)(k * 2),
-                     idesc, (kb | k) != 0 ? 1u : 0u);
+            const uint32_t td = tacc + (uint32_t)(j * a.BN);
+            if (ksteps == 4) {
+              mma_i8(td, da, db, idesc, kb != 0 ? 1u : 0u);
+              mma_i8(td, da + 2u, db + 2u, idesc, 1u);
+              mma_i8(td, da + 4u, db + 4u, idesc, 1u);
+              mma_i8(td, da + 6u, db + 6u, idesc, 1u);
+            } else {
+              for (int k = 0; k < ksteps; ++k)
+                mma_i8(td, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+            }
           }
           mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
           if (++s == a.stages) { s = 0; ph ^= 1u; }

@@ -367,7 +367,12 @@ int forward_impl(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float
     const CUtensorMap* mx = map_x(pl, x);
     const CUtensorMap* mv = map_stage(pl, pl->cache_vst, Vq, pl->p.C);
     if (mx == nullptr || mv == nullptr) return WINO_ERR_CUDA;
-    rc = launch_input_transform_tma(pl->p, opt_of(pl, pdl), *mx, *mv, pl->status_dev, st);
+    LaunchOpt o = opt_of(pl, pdl);
+    if ((stage_mask & 2) && !calib) {   // the GEMMs that follow read U_q, which no kernel of this call writes
+      o.l2_hint = Uq;
+      o.l2_hint_bytes = (size_t)pl->p.t * pl->p.t * pl->p.K * pl->p.C;
+    }
+    rc = launch_input_transform_tma(pl->p, o, *mx, *mv, pl->status_dev, st);
   } else {
     rc = launch_input_transform(pl->p, opt_of(pl, pdl), x, Vq, calib ? absmax4 + 0 : nullptr, st);
   }

@@ -16,6 +16,11 @@ struct LaunchOpt {
   bool std_mats = false;      // B^T and A^T are the built-in Cook-Toom matrices
   bool pdl = false;           // programmatic dependent launch on the stream
   int device = 0;             // the plan's device (current when the launcher runs)
+  // A buffer a later kernel of the same call will read and that no kernel of the call
+  // writes (the transformed weights): the input transform's blocks ask for it to be brought
+  // into L2 while they run.  A hint only; null: none.
+  const void* l2_hint = nullptr;
+  size_t l2_hint_bytes = 0;   // a multiple of 16
 };
 
 // "Done once per device" bookkeeping.  cudaFuncSetAttribute applies to the device

@@ -146,6 +146,17 @@ __device__ __forceinline__ void tma_prefetch_l2_4d(const CUtensorMap* map, int c
   asm volatile("cp.async.bulk.prefetch.tensor.4d.L2.global.tile [%0, {%1, %2, %3, %4}];"
                ::"l"(map), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
 }
+// Hint: bring `bytes` (a multiple of 16) at a 16-byte aligned global address into L2.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* gptr, uint32_t bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(gptr), "r"(bytes) : "memory");
+}
+// This block's share of a buffer that the whole grid is asked to bring into L2.
+__device__ __forceinline__ void l2_hint_slice(const uint8_t* base, uint32_t total_bytes) {
+  if (base == nullptr) return;
+  const uint32_t per = ((total_bytes + gridDim.x - 1) / gridDim.x + 15u) & ~15u;
+  const uint32_t off = blockIdx.x * per;
+  if (off < total_bytes) bulk_prefetch_l2(base + off, min(per, total_bytes - off));
+}
 __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c0, int c1, int c2) {
   asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global.tile [%0, {%1, %2, %3}];"
                ::"l"(map), "r"(c0), "r"(c1), "r"(c2) : "memory");

@@ -8,7 +8,7 @@
 
 #ifdef WINO_TRACE
 namespace wino {
-constexpr int kTraceSteps = 32, kTraceBlocks = 2368, kTraceSlots = 12;
+constexpr int kTraceSteps = 32, kTraceBlocks = 2368, kTraceSlots = 16;
 struct TraceTable {
   unsigned long long t[kTraceSteps][kTraceBlocks][kTraceSlots];
   unsigned int launches[kTraceBlocks];

@@ -50,7 +50,8 @@ WINO_ST_READER(wino_trace_output, g_out_trace)
 template <int M, int MODE, int CC, int G, int CPT>
 __global__ void __launch_bounds__((CC / CPT) * G)
 k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
-                      const __grid_constant__ CUtensorMap mapV, int* __restrict__ status) {
+                      const __grid_constant__ CUtensorMap mapV, int* __restrict__ status,
+                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
   constexpr uint32_t kTileStride = (kTileBytes + 127u) & ~127u;   // TMA destinations stay 128-byte aligned
@@ -92,6 +93,7 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
       tma_prefetch_l2_4d(&mapX, c0, (tau % p.TW) * M - 1, ((tau / p.TW) % p.TH) * M - 1,
                          tau / (p.TW * p.TH));
     }
+    l2_hint_slice(l2_hint, l2_hint_bytes);   // what the next kernel will want from HBM
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
     WINO_ST(g_in_trace, trace_step, 1);
     mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
@@ -159,7 +161,8 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
 template <int M, int MODE, int CC, int G, int CPT, int UPB>
 __global__ void __launch_bounds__((CC / CPT) * G)
 k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
-                            const __grid_constant__ CUtensorMap mapV, int* __restrict__ status) {
+                            const __grid_constant__ CUtensorMap mapV, int* __restrict__ status,
+                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
   constexpr uint32_t kTileStride = (kTileBytes + 127u) & ~127u;
@@ -197,6 +200,7 @@ k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_const
   if (threadIdx.x == 0) {
     tma_prefetch_map(&mapX);
     tma_prefetch_map(&mapV);
+    l2_hint_slice(l2_hint, l2_hint_bytes);
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
 #pragma unroll
     for (int r = 0; r < UPB; ++r)
@@ -386,7 +390,8 @@ int input_tma_launch_u(const Params& p, const LaunchOpt& o, const CUtensorMap& m
   if (int rc = set_max_smem(once, o.device, kernel, smem)) return rc;
   const int units = ((p.T + G - 1) / G) * (p.C / CC);
   return launch_kernel(kernel, dim3((unsigned)((units + UPB - 1) / UPB)), dim3((CC / CPT) * G), smem,
-                       st, o.pdl, p, mapX, mapV, status);
+                       st, o.pdl, p, mapX, mapV, status, static_cast<const uint8_t*>(o.l2_hint),
+                       (uint32_t)o.l2_hint_bytes);
 }
 template <int M, int MODE, int CC, int G, int CPT>
 int input_tma_launch(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX, const CUtensorMap& mapV,
