@@ -197,9 +197,14 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
 }
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
-k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV,
-          const __grid_constant__ CUtensorMap mapU, const GemmTcArgs a, void* __restrict__ out,
+k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV_param,
+          const __grid_constant__ CUtensorMap mapU_param, const CUtensorMap* __restrict__ devV,
+          const CUtensorMap* __restrict__ devU, const GemmTcArgs a, void* __restrict__ out,
           unsigned* __restrict__ absmaxM, int* __restrict__ status) {
+  // device-resident descriptors when the plan has them (warm, and prefetched by the kernel
+  // before this one), else the copies in the parameter buffer
+  const CUtensorMap* mapV = devV != nullptr ? devV : &mapV_param;
+  const CUtensorMap* mapU = devU != nullptr ? devU : &mapU_param;
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -240,9 +245,6 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     }
     *abort_p = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-#ifdef WINO_TRACE
-    WINO_ST(g_gemm_trace, trace_step_s, 12);
-#endif
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, (uint32_t)a.tmem_cols);
@@ -251,14 +253,9 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
 #endif
   }
   if (warp == 0 && lane == 0) {   // descriptors do not depend on the previous kernel
-    tma_prefetch_map(&mapV);
-    tma_prefetch_map(&mapU);
-#ifdef WINO_TRACE
-    WINO_ST(g_gemm_trace, trace_step_s, 14);
-#endif
-#ifdef WINO_TRACE
-    WINO_ST(g_gemm_trace, trace_step_s, 15);
-#endif
+    tma_prefetch_map(mapV);
+    tma_prefetch_map(mapU);
+
   }
   tc_fence_before();
   __syncthreads();
@@ -271,25 +268,34 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     g_gemm_trace.t[trace_step][blockIdx.x][13] = *reinterpret_cast<unsigned long long*>(gen + (tmem_slot + 16u - base));
   }
 #endif
-  griddep_wait();   // everything below reads or writes buffers other kernels touch
-  if (threadIdx.x == 0) WINO_ST(g_gemm_trace, trace_step, 2);
-
+  // Each role waits for the preceding kernels itself, as late as it can: the producer just
+  // before its first load (its index arithmetic is done by then), the epilogue warps before
+  // they write; the MMA thread touches no global memory.
   if (warp == 0) {
     if (lane == 0) {
-      int s = 0; uint32_t ph = 0;
+      int s = 0, issued = 0; uint32_t ph = 0;
+      int xi = blockIdx.x / per_xi, rem = blockIdx.x - xi * per_xi;
+      int nb = rem / a.n_mblk, mb = rem - nb * a.n_mblk;
+      griddep_wait();
+      WINO_ST(g_gemm_trace, trace_step, 2);
       for (int it = blockIdx.x; it < a.n_items; it += gridDim.x) {
-        const int xi = it / per_xi, rem = it - xi * per_xi;
-        const int nb = rem / a.n_mblk, mb = rem - nb * a.n_mblk;
+        if (it != blockIdx.x) {
+          xi = it / per_xi; rem = it - xi * per_xi;
+          nb = rem / a.n_mblk; mb = rem - nb * a.n_mblk;
+        }
         bool ok = true;
         for (int kb = 0; kb < KB; ++kb) {
-          if (!mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
+          // the ring's first pass finds every stage free
+          if (issued >= a.stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
+          ++issued;
           const uint32_t sa = base + (uint32_t)s * stage_bytes;
           mbar_expect_tx(bar_full + 8u * s, stage_bytes);
           for (int j = 0; j < a.MB; ++j)   // rows past T are filled with zeros by the TMA unit
-            tma_load_3d(sa + (uint32_t)j * a_bytes, &mapV, bar_full + 8u * s, kb * kStageK,
+            tma_load_3d(sa + (uint32_t)j * a_bytes, mapV, bar_full + 8u * s, kb * kStageK,
                         (mb * a.MB + j) * kBM, xi);
-          tma_load_3d(sa + (uint32_t)a.MB * a_bytes, &mapU, bar_full + 8u * s, kb * kStageK,
+          tma_load_3d(sa + (uint32_t)a.MB * a_bytes, mapU, bar_full + 8u * s, kb * kStageK,
                       nb * a.BN, xi);
+          if (it == blockIdx.x && kb == 0) WINO_ST(g_gemm_trace, trace_step, 15);
           if (++s == a.stages) { s = 0; ph ^= 1u; }
         }
         if (!ok) { *abort_p = 1u; break; }
@@ -343,6 +349,7 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     // of every column block lies inside K (the last block is not ragged).
     const bool small = p.C <= 260;
     const bool full = (p.K % a.BN) == 0 && (a.BN % 32) == 0;
+    griddep_wait();
     if (absmaxM != nullptr)
       epilogue_loop<false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
                                         abort_p, warp, lane, trace_step);
@@ -393,8 +400,8 @@ TcGeom tc_geometry(const Params& p, int num_sms) {
 }
 
 int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,
-                   const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
-                   int* status, cudaStream_t st) {
+                   const CUtensorMap& mapU, const CUtensorMap* devV, const CUtensorMap* devU,
+                   void* out, int out_mode, unsigned* absmaxM, int* status, cudaStream_t st) {
   static DeviceOnce once;
   if (int rc = set_max_smem(once, o.device, k_gemm_tc, 227 * 1024)) return rc;
   GemmTcArgs a;
@@ -405,7 +412,7 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
   a.n_nblk = (p.K + g.BN - 1) / g.BN;
   a.n_items = p.t * p.t * a.n_mblk * a.n_nblk;
   return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,
-                       mapV, mapU, a, out, absmaxM, status);
+                       mapV, mapU, devV, devU, a, out, absmaxM, status);
 }
 
 }  // namespace wino

@@ -47,11 +47,22 @@ WINO_ST_READER(wino_trace_input, g_in_trace)
 WINO_ST_READER(wino_trace_output, g_out_trace)
 #endif
 
-template <int M, int MODE, int CC, int G, int CPT>
-__global__ void __launch_bounds__((CC / CPT) * G)
+// Blocks per SM asked of the compiler.  One channel per thread: a full SM of threads (2048),
+// i.e. at most 32 registers each.  The output transform fits that without spilling.  The input
+// transform does not (it spills some sixty words), so it exists in two builds and the launcher
+// takes the 32-register one only where it turns a grid of slightly more than one wave into a
+// single wave: the 2048 blocks of a 256-channel, 1024-tile layer are then resident together,
+// where otherwise a second, nearly empty wave lengthened the kernel by a quarter.
+constexpr int tma_min_blocks(int threads, int cpt, bool cap) {
+  return (cpt == 1 && cap) ? (2048 / threads > 32 ? 32 : 2048 / threads) : 1;
+}
+
+template <int M, int MODE, int CC, int G, int CPT, bool CAP>
+__global__ void __launch_bounds__((CC / CPT) * G, tma_min_blocks((CC / CPT) * G, CPT, CAP))
 k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
                       const __grid_constant__ CUtensorMap mapV, int* __restrict__ status,
-                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes) {
+                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes,
+                      const CUtensorMap* __restrict__ next0, const CUtensorMap* __restrict__ next1) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
   constexpr uint32_t kTileStride = (kTileBytes + 127u) & ~127u;   // TMA destinations stay 128-byte aligned
@@ -86,24 +97,29 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
   if (threadIdx.x == 0) {
     tma_prefetch_map(&mapX);
     tma_prefetch_map(&mapV);
+    // patch coordinates first: nothing but the loads themselves is left for after the wait
+    int cw[G], ch[G], cn[G];
+#pragma unroll
+    for (int i = 0; i < G; ++i) {
+      const int tau = tau0 + i;
+      cw[i] = (tau % p.TW) * M - 1;
+      ch[i] = ((tau / p.TW) % p.TH) * M - 1;
+      cn[i] = tau / (p.TW * p.TH);
+    }
     // ask for the patches to be brought into L2 while the preceding kernel is still running
     // (a hint only: nothing is read into the SM before the wait below)
-    for (int i = 0; i < ntile; ++i) {
-      const int tau = tau0 + i;
-      tma_prefetch_l2_4d(&mapX, c0, (tau % p.TW) * M - 1, ((tau / p.TW) % p.TH) * M - 1,
-                         tau / (p.TW * p.TH));
-    }
+#pragma unroll
+    for (int i = 0; i < G; ++i)
+      if (i < ntile) tma_prefetch_l2_4d(&mapX, c0, cw[i], ch[i], cn[i]);
     l2_hint_slice(l2_hint, l2_hint_bytes);   // what the next kernel will want from HBM
+    if (next0 != nullptr) tma_prefetch_map(next0);   // ... and its descriptors
+    if (next1 != nullptr) tma_prefetch_map(next1);
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
     WINO_ST(g_in_trace, trace_step, 1);
     mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
-    for (int i = 0; i < ntile; ++i) {
-      const int tau = tau0 + i;
-      const int tw = tau % p.TW;
-      const int th = (tau / p.TW) % p.TH;
-      const int n = tau / (p.TW * p.TH);
-      tma_load_4d(s_in + (uint32_t)i * kTileStride, &mapX, bar, c0, tw * M - 1, th * M - 1, n);
-    }
+#pragma unroll
+    for (int i = 0; i < G; ++i)
+      if (i < ntile) tma_load_4d(s_in + (uint32_t)i * kTileStride, &mapX, bar, c0, cw[i], ch[i], cn[i]);
     // one thread polls (bounded); the others sleep in the barrier below
     if (!mbar_wait(bar, 0u, &abort_flag)) {
       abort_flag = 1u;
@@ -162,7 +178,8 @@ template <int M, int MODE, int CC, int G, int CPT, int UPB>
 __global__ void __launch_bounds__((CC / CPT) * G)
 k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
                             const __grid_constant__ CUtensorMap mapV, int* __restrict__ status,
-                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes) {
+                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes,
+                      const CUtensorMap* __restrict__ next0, const CUtensorMap* __restrict__ next1) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
   constexpr uint32_t kTileStride = (kTileBytes + 127u) & ~127u;
@@ -201,6 +218,8 @@ k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_const
     tma_prefetch_map(&mapX);
     tma_prefetch_map(&mapV);
     l2_hint_slice(l2_hint, l2_hint_bytes);
+    if (next0 != nullptr) tma_prefetch_map(next0);
+    if (next1 != nullptr) tma_prefetch_map(next1);
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
 #pragma unroll
     for (int r = 0; r < UPB; ++r)
@@ -263,7 +282,7 @@ k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_const
 }
 
 template <int M, int MODE, int KC, int G, int CPT>
-__global__ void __launch_bounds__((KC / CPT) * G)
+__global__ void __launch_bounds__((KC / CPT) * G, tma_min_blocks((KC / CPT) * G, CPT, true))
 k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapM,
                        const __grid_constant__ CUtensorMap mapY, const float* __restrict__ bias,
                        float s_Y, int* __restrict__ status) {
@@ -379,19 +398,55 @@ inline int tma_cpt(long tiles_times_channels) {
   return tiles_times_channels / (4 * 32) >= 148l * 64 ? 4 : 1;
 }
 
+// Resident blocks per SM of a kernel, asked once per instantiation and device.
+template <auto kernel>
+int resident_blocks(int threads, size_t smem, int device) {
+  static std::mutex mu;
+  static int cache[64];   // 0: not asked yet
+  std::lock_guard<std::mutex> lock(mu);
+  const int d = device >= 0 && device < 64 ? device : 0;
+  if (cache[d] == 0) {
+    int nb = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&nb, kernel, threads, smem) != cudaSuccess || nb < 1) {
+      cudaGetLastError();
+      nb = 1;
+    }
+    cache[d] = nb;
+  }
+  return cache[d];
+}
+
 template <int M, int MODE, int CC, int G, int CPT, int UPB>
 int input_tma_launch_u(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX, const CUtensorMap& mapV,
                        int* status, cudaStream_t st) {
   constexpr size_t smem =
       2 * (size_t)UPB * G * ((((M + 2) * (M + 2) * CC) + 127) / 128 * 128) + 128 + 16 * UPB;
-  auto kernel = UPB == 1 ? k_input_transform_tma<M, MODE, CC, G, CPT>
-                         : k_input_transform_tma_multi<M, MODE, CC, G, CPT, UPB>;
-  static DeviceOnce once;   // one per instantiation
-  if (int rc = set_max_smem(once, o.device, kernel, smem)) return rc;
+  constexpr int threads = (CC / CPT) * G;
   const int units = ((p.T + G - 1) / G) * (p.C / CC);
-  return launch_kernel(kernel, dim3((unsigned)((units + UPB - 1) / UPB)), dim3((CC / CPT) * G), smem,
-                       st, o.pdl, p, mapX, mapV, status, static_cast<const uint8_t*>(o.l2_hint),
-                       (uint32_t)o.l2_hint_bytes);
+  if constexpr (UPB == 1 && CPT == 1) {
+    // the 32-register build only where it saves a second wave
+    static DeviceOnce once_a, once_b;
+    auto ka = k_input_transform_tma<M, MODE, CC, G, CPT, false>;
+    auto kb = k_input_transform_tma<M, MODE, CC, G, CPT, true>;
+    if (int rc = set_max_smem(once_a, o.device, ka, smem)) return rc;
+    if (int rc = set_max_smem(once_b, o.device, kb, smem)) return rc;
+    const int na = resident_blocks<k_input_transform_tma<M, MODE, CC, G, CPT, false>>(threads, smem, o.device) * o.num_sms;
+    const int nb = resident_blocks<k_input_transform_tma<M, MODE, CC, G, CPT, true>>(threads, smem, o.device) * o.num_sms;
+    const bool cap = units > na && units <= nb;
+    return launch_kernel(cap ? kb : ka, dim3((unsigned)units), dim3(threads), smem, st, o.pdl, p, mapX,
+                         mapV, status, static_cast<const uint8_t*>(o.l2_hint), (uint32_t)o.l2_hint_bytes,
+                         o.next_maps[0], o.next_maps[1]);
+  } else {
+    auto kernel = [] {
+      if constexpr (UPB == 1) return k_input_transform_tma<M, MODE, CC, G, CPT, false>;
+      else return k_input_transform_tma_multi<M, MODE, CC, G, CPT, UPB>;
+    }();
+    static DeviceOnce once;   // one per instantiation
+    if (int rc = set_max_smem(once, o.device, kernel, smem)) return rc;
+    return launch_kernel(kernel, dim3((unsigned)((units + UPB - 1) / UPB)), dim3(threads), smem, st, o.pdl,
+                         p, mapX, mapV, status, static_cast<const uint8_t*>(o.l2_hint),
+                         (uint32_t)o.l2_hint_bytes, o.next_maps[0], o.next_maps[1]);
+  }
 }
 template <int M, int MODE, int CC, int G, int CPT>
 int input_tma_launch(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX, const CUtensorMap& mapV,
