@@ -302,31 +302,33 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
       }
     }
   } else if (warp == 1) {
-    if (lane == 0) {
-      const uint32_t idesc = make_idesc_i8(kBM, a.BN);
-      int s = 0; uint32_t ph = 0;
-      int li = 0;
-      for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
-        const int buf = li & 1;
-        const uint32_t aph = (uint32_t)(li >> 1) & 1u;
-        bool ok = mbar_wait(bar_acc_empty + 8u * buf, aph ^ 1u, abort_p);
+    // The whole warp walks the loop so that stage addresses and descriptors are warp-uniform
+    // values; one elected lane issues the MMAs and the commits.
+    const bool leader = elect_one();
+    const uint32_t idesc = make_idesc_i8(kBM, a.BN);
+    int s = 0; uint32_t ph = 0;
+    int li = 0;
+    for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
+      const int buf = li & 1;
+      const uint32_t aph = (uint32_t)(li >> 1) & 1u;
+      bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8u * buf, aph ^ 1u, abort_p));
+      tc_fence_after();
+      const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride);
+      for (int kb = 0; kb < KB && ok; ++kb) {
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph, abort_p))) { ok = false; break; }
+        if (leader && li == 0 && kb == 0) WINO_ST(g_gemm_trace, trace_step, 3);
+        if (leader && li == 0 && kb == KB - 1) WINO_ST(g_gemm_trace, trace_step, 4);
+        if (leader && li == 1 && kb == 0) WINO_ST(g_gemm_trace, trace_step, 10);
+        if (leader && li == 1 && kb == KB - 1) WINO_ST(g_gemm_trace, trace_step, 11);
         tc_fence_after();
-        const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride);
-        for (int kb = 0; kb < KB && ok; ++kb) {
-          if (!mbar_wait(bar_full + 8u * s, ph, abort_p)) { ok = false; break; }
-          if (li == 0 && kb == 0) WINO_ST(g_gemm_trace, trace_step, 3);
-          if (li == 0 && kb == KB - 1) WINO_ST(g_gemm_trace, trace_step, 4);
-          if (li == 1 && kb == 0) WINO_ST(g_gemm_trace, trace_step, 10);
-          if (li == 1 && kb == KB - 1) WINO_ST(g_gemm_trace, trace_step, 11);
-          tc_fence_after();
-          const uint32_t sa = base + (uint32_t)s * stage_bytes;
-          const uint64_t db = make_desc_sw128(sa + (uint32_t)a.MB * a_bytes);
-          const int remc = p.C - kb * kStageK;
-          const int ksteps = remc >= kStageK ? 4 : (remc + 31) / 32;
-          // (few instructions per MMA: this thread shares its scheduler with epilogue warps)
-          for (int j = 0; j < a.MB; ++j) {
-            const uint64_t da = make_desc_sw128(sa + (uint32_t)j * a_bytes);
-            const uint32_t td = tacc + (uint32_t)(j * a.BN);
+        const uint32_t sa = base + (uint32_t)s * stage_bytes;
+        const uint64_t db = make_desc_sw128(sa + (uint32_t)a.MB * a_bytes);
+        const int remc = p.C - kb * kStageK;
+        const int ksteps = remc >= kStageK ? 4 : (remc + 31) / 32;
+        for (int j = 0; j < a.MB; ++j) {
+          const uint64_t da = make_desc_sw128(sa + (uint32_t)j * a_bytes);
+          const uint32_t td = tacc + (uint32_t)(j * a.BN);
+          if (leader) {
             if (ksteps == 4) {
               mma_i8(td, da, db, idesc, kb != 0 ? 1u : 0u);
               mma_i8(td, da + 2u, db + 2u, idesc, 1u);
@@ -337,12 +339,14 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
                 mma_i8(td, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (kb | k) != 0 ? 1u : 0u);
             }
           }
-          mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
-          if (++s == a.stages) { s = 0; ph ^= 1u; }
         }
-        if (!ok) { *abort_p = 1u; break; }
-        mma_commit(bar_acc_full + 8u * buf);  // accumulator complete
+        if (leader) mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
+        __syncwarp();
+        if (++s == a.stages) { s = 0; ph ^= 1u; }
       }
+      if (!ok) { *abort_p = 1u; break; }
+      if (leader) mma_commit(bar_acc_full + 8u * buf);  // accumulator complete
+      __syncwarp();
     }
   } else {
     // epilogue warps.  small: |M| <= 127^2 * C < 2^22; full: every 32-column chunk

@@ -57,6 +57,18 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
     }
   }
 }
+// One lane of a fully active warp (the same one every time it is asked).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t is_leader;
+  asm volatile(
+      "{\n"
+      ".reg .pred p;\n"
+      "elect.sync _|p, 0xffffffff;\n"
+      "selp.u32 %0, 1, 0, p;\n"
+      "}\n"
+      : "=r"(is_leader));
+  return is_leader != 0u;
+}
 // Fetch a tensor map into the descriptor cache ahead of its first use.
 __device__ __forceinline__ void tma_prefetch_map(const CUtensorMap* map) {
   asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
