@@ -198,13 +198,10 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV_param,
-          const __grid_constant__ CUtensorMap mapU_param, const CUtensorMap* __restrict__ devV,
-          const CUtensorMap* __restrict__ devU, const GemmTcArgs a, void* __restrict__ out,
+          const __grid_constant__ CUtensorMap mapU_param, const GemmTcArgs a, void* __restrict__ out,
           unsigned* __restrict__ absmaxM, int* __restrict__ status) {
-  // device-resident descriptors when the plan has them (warm, and prefetched by the kernel
-  // before this one), else the copies in the parameter buffer
-  const CUtensorMap* mapV = devV != nullptr ? devV : &mapV_param;
-  const CUtensorMap* mapU = devU != nullptr ? devU : &mapU_param;
+  const CUtensorMap* mapV = &mapV_param;
+  const CUtensorMap* mapU = &mapU_param;
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -404,8 +401,8 @@ TcGeom tc_geometry(const Params& p, int num_sms) {
 }
 
 int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,
-                   const CUtensorMap& mapU, const CUtensorMap* devV, const CUtensorMap* devU,
-                   void* out, int out_mode, unsigned* absmaxM, int* status, cudaStream_t st) {
+                   const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
+                   int* status, cudaStream_t st) {
   static DeviceOnce once;
   if (int rc = set_max_smem(once, o.device, k_gemm_tc, 227 * 1024)) return rc;
   GemmTcArgs a;
@@ -416,7 +413,7 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
   a.n_nblk = (p.K + g.BN - 1) / g.BN;
   a.n_items = p.t * p.t * a.n_mblk * a.n_nblk;
   return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,
-                       mapV, mapU, devV, devU, a, out, absmaxM, status);
+                       mapV, mapU, a, out, absmaxM, status);
 }
 
 }  // namespace wino

@@ -48,17 +48,6 @@ struct wino_plan {
   int* status_dev;      // device status word (may be null when no GPU is present)
   void* kron_dev;       // Kronecker tables of the tensor-core transforms (same allocation)
   unsigned* counters_dev;  // progress counters of the single-launch layer kernel (same allocation)
-  // Device-resident copies of tensor maps (same allocation), keyed by (kind, base address).
-  // A CTA that starts late (the GEMM's, which wait for the shared memory of the kernel before
-  // them) would otherwise stall its first TMA loads on fetching descriptors from a cold
-  // parameter buffer; descriptors at a fixed device address stay warm and can be
-  // prefetched by the preceding kernel.  Entries are never replaced (a captured graph may
-  // replay the upload of one); when the table is full the parameter copy is used.
-  CUtensorMap* maps_dev;
-  CUtensorMap* maps_pinned;
-  const void* map_keys[kDevMaps];
-  int map_kinds[kDevMaps];
-  int maps_used;
   CUtensorMap fmapV, fmapU;   // GEMM operand maps of the single-launch kernel
   const void* fmap_vq_ptr;
   const void* fmap_uq_ptr;
@@ -163,25 +152,6 @@ bool path_supported(const wino_plan_t* pl, int path) {
 size_t vq_bytes(const wino_plan_t* pl) { return (size_t)pl->p.t * pl->p.t * pl->p.T * pl->p.C; }
 size_t m_elems(const wino_plan_t* pl) { return (size_t)pl->p.t * pl->p.t * pl->p.T * pl->p.K; }
 size_t mbuf_bytes(const wino_plan_t* pl) { return m_elems(pl) * (pl->p.qM_enabled ? 1 : 4); }
-
-const CUtensorMap* dev_map(wino_plan_t* pl, int kind, const void* key, const CUtensorMap& host,
-                           cudaStream_t st) {
-  if (pl->maps_dev == nullptr || pl->maps_pinned == nullptr) return nullptr;
-  for (int i = 0; i < pl->maps_used; ++i)
-    if (pl->map_keys[i] == key && pl->map_kinds[i] == kind) return pl->maps_dev + i;
-  if (pl->maps_used >= kDevMaps) return nullptr;
-  const int i = pl->maps_used;
-  pl->maps_pinned[i] = host;
-  if (cudaMemcpyAsync(pl->maps_dev + i, pl->maps_pinned + i, sizeof(CUtensorMap),
-                      cudaMemcpyHostToDevice, st) != cudaSuccess) {
-    cudaGetLastError();
-    return nullptr;
-  }
-  pl->map_keys[i] = key;
-  pl->map_kinds[i] = kind;
-  pl->maps_used = i + 1;
-  return pl->maps_dev + i;
-}
 
 LaunchOpt opt_of(const wino_plan_t* pl, bool pdl) {
   LaunchOpt o;
@@ -299,12 +269,13 @@ const CUtensorMap* map_u_fused(wino_plan_t* pl, const void* Uq) {
   return m;
 }
 
-// The GEMM's operand maps for these buffers: host copies in the plan, device copies if the
-// table has room (uploaded on `st` the first time a buffer is seen).
-int gemm_maps(wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, cudaStream_t st,
-              const CUtensorMap** dV, const CUtensorMap** dU) {
+int launch_gemm(wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void* out, int out_mode,
+                unsigned* absmaxM, bool pdl, cudaStream_t st) {
   const Params& p = pl->p;
   const int t2 = p.t * p.t;
+  pl->launches++;
+  if (pl->path == WINO_PATH_STAGED_DP4A)
+    return launch_gemm_dp4a(p, opt_of(pl, pdl), Vq, Uq, out, out_mode, absmaxM, st);
   const TcGeom g = tc_geometry(p, pl->num_sms);
   if (pl->map_vq_ptr != Vq) {
     int rc = encode_map(&pl->mapV, Vq, (uint64_t)p.C, (uint64_t)p.T, (uint64_t)t2, kBM);
@@ -316,21 +287,7 @@ int gemm_maps(wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, cudaStream_t 
     if (rc != WINO_OK) return rc;
     pl->map_uq_ptr = Uq;
   }
-  *dV = dev_map(pl, 0, Vq, pl->mapV, st);
-  *dU = dev_map(pl, 1, Uq, pl->mapU, st);
-  return WINO_OK;
-}
-
-int launch_gemm(wino_plan_t* pl, const int8_t* Vq, const int8_t* Uq, void* out, int out_mode,
-                unsigned* absmaxM, bool pdl, cudaStream_t st) {
-  const Params& p = pl->p;
-  pl->launches++;
-  if (pl->path == WINO_PATH_STAGED_DP4A)
-    return launch_gemm_dp4a(p, opt_of(pl, pdl), Vq, Uq, out, out_mode, absmaxM, st);
-  const TcGeom g = tc_geometry(p, pl->num_sms);
-  const CUtensorMap *dV = nullptr, *dU = nullptr;
-  if (int rc = gemm_maps(pl, Vq, Uq, st, &dV, &dU)) return rc;
-  return launch_gemm_tc(p, opt_of(pl, pdl), g, pl->mapV, pl->mapU, dV, dU, out, out_mode, absmaxM,
+  return launch_gemm_tc(p, opt_of(pl, pdl), g, pl->mapV, pl->mapU, out, out_mode, absmaxM,
                         pl->status_dev, st);
 }
 
@@ -415,8 +372,6 @@ int forward_impl(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float
     if ((stage_mask & 2) && !calib) {   // the GEMMs that follow read U_q, which no kernel of this call writes
       o.l2_hint = Uq;
       o.l2_hint_bytes = (size_t)pl->p.t * pl->p.t * pl->p.K * pl->p.C;
-      if (gemm_maps(pl, Vq, Uq, st, &o.next_maps[0], &o.next_maps[1]) != WINO_OK)
-        o.next_maps[0] = o.next_maps[1] = nullptr;
     }
     rc = launch_input_transform_tma(pl->p, o, *mx, *mv, pl->status_dev, st);
   } else {
@@ -539,16 +494,11 @@ int wino_plan(const wino_desc_t* desc, wino_plan_t** out) {
         sms > 0)
       pl->num_sms = sms;
     // one small allocation: the status word, then (256 bytes in) the Kronecker tables
-    const size_t maps_off = (256 + kKronBytes + sizeof(unsigned) * kFusedCounterWords + 127) / 128 * 128;
-    const size_t dev_bytes = maps_off + sizeof(CUtensorMap) * kDevMaps;
+    const size_t dev_bytes = 256 + kKronBytes + sizeof(unsigned) * kFusedCounterWords;
     if (cudaMalloc(&pl->status_dev, dev_bytes) == cudaSuccess) {
       cudaMemset(pl->status_dev, 0, dev_bytes);
       pl->kron_dev = reinterpret_cast<uint8_t*>(pl->status_dev) + 256;
       pl->counters_dev = reinterpret_cast<unsigned*>(reinterpret_cast<uint8_t*>(pl->kron_dev) + kKronBytes);
-      pl->maps_dev = reinterpret_cast<CUtensorMap*>(reinterpret_cast<uint8_t*>(pl->status_dev) + maps_off);
-      void* pinned = nullptr;
-      if (cudaMallocHost(&pinned, sizeof(CUtensorMap) * kDevMaps) == cudaSuccess)
-        pl->maps_pinned = static_cast<CUtensorMap*>(pinned);
       if (pl->std_mats && (d.m == 2 || d.m == 4)) {
         int8_t tables[kKronBytes];
         fill_kronecker_tables(d.m, tables);
@@ -745,7 +695,6 @@ long wino_launch_count(const wino_plan_t* pl) { return pl ? pl->launches : 0; }
 void wino_destroy(wino_plan_t* pl) {
   if (pl == nullptr) return;
   if (pl->status_dev) cudaFree(pl->status_dev);
-  if (pl->maps_pinned) cudaFreeHost(pl->maps_pinned);
   delete pl;
 }
 

@@ -22,11 +22,7 @@ struct LaunchOpt {
   // into L2 while they run.  A hint only; null: none.
   const void* l2_hint = nullptr;
   size_t l2_hint_bytes = 0;   // a multiple of 16
-  // Device-resident tensor maps the next kernel will use (null: none): the input transform's
-  // blocks prefetch them into the descriptor cache.
-  const CUtensorMap* next_maps[2] = {nullptr, nullptr};
 };
-constexpr int kDevMaps = 96;   // device-resident tensor maps per plan
 
 // "Done once per device" bookkeeping.  cudaFuncSetAttribute applies to the device
 // that is current when it is called, so the opt-in to more than 48 KB of dynamic
@@ -121,8 +117,8 @@ int launch_layer_fused(const Params& p, const LaunchOpt& o, const FusedGeom& g, 
 struct TcGeom { int BN, MB, stages, tmem_cols, grid; size_t smem; };
 TcGeom tc_geometry(const Params& p, int num_sms);
 int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const CUtensorMap& mapV,
-                   const CUtensorMap& mapU, const CUtensorMap* devV, const CUtensorMap* devU,
-                   void* out, int out_mode, unsigned* absmaxM, int* status, cudaStream_t st);
+                   const CUtensorMap& mapU, void* out, int out_mode, unsigned* absmaxM,
+                   int* status, cudaStream_t st);
 int launch_smallc(const Params& p, const LaunchOpt& o, const int8_t* x, const int8_t* Uq,
                   const float* bias, void* y, float s_Y, int* dbgM, cudaStream_t st);
 

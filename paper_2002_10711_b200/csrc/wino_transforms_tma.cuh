@@ -61,8 +61,7 @@ template <int M, int MODE, int CC, int G, int CPT, bool CAP>
 __global__ void __launch_bounds__((CC / CPT) * G, tma_min_blocks((CC / CPT) * G, CPT, CAP))
 k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
                       const __grid_constant__ CUtensorMap mapV, int* __restrict__ status,
-                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes,
-                      const CUtensorMap* __restrict__ next0, const CUtensorMap* __restrict__ next1) {
+                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
   constexpr uint32_t kTileStride = (kTileBytes + 127u) & ~127u;   // TMA destinations stay 128-byte aligned
@@ -112,8 +111,6 @@ k_input_transform_tma(const __grid_constant__ Params p, const __grid_constant__ 
     for (int i = 0; i < G; ++i)
       if (i < ntile) tma_prefetch_l2_4d(&mapX, c0, cw[i], ch[i], cn[i]);
     l2_hint_slice(l2_hint, l2_hint_bytes);   // what the next kernel will want from HBM
-    if (next0 != nullptr) tma_prefetch_map(next0);   // ... and its descriptors
-    if (next1 != nullptr) tma_prefetch_map(next1);
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
     WINO_ST(g_in_trace, trace_step, 1);
     mbar_expect_tx(bar, (uint32_t)ntile * kTileBytes);
@@ -178,8 +175,7 @@ template <int M, int MODE, int CC, int G, int CPT, int UPB>
 __global__ void __launch_bounds__((CC / CPT) * G)
 k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapX,
                             const __grid_constant__ CUtensorMap mapV, int* __restrict__ status,
-                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes,
-                      const CUtensorMap* __restrict__ next0, const CUtensorMap* __restrict__ next1) {
+                      const uint8_t* __restrict__ l2_hint, uint32_t l2_hint_bytes) {
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = CC / CPT;
   constexpr uint32_t kTileBytes = T2 * CC;
   constexpr uint32_t kTileStride = (kTileBytes + 127u) & ~127u;
@@ -218,8 +214,6 @@ k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_const
     tma_prefetch_map(&mapX);
     tma_prefetch_map(&mapV);
     l2_hint_slice(l2_hint, l2_hint_bytes);
-    if (next0 != nullptr) tma_prefetch_map(next0);
-    if (next1 != nullptr) tma_prefetch_map(next1);
     griddep_wait();   // only this thread reads or writes buffers that other kernels touch
 #pragma unroll
     for (int r = 0; r < UPB; ++r)
@@ -434,8 +428,7 @@ int input_tma_launch_u(const Params& p, const LaunchOpt& o, const CUtensorMap& m
     const int nb = resident_blocks<k_input_transform_tma<M, MODE, CC, G, CPT, true>>(threads, smem, o.device) * o.num_sms;
     const bool cap = units > na && units <= nb;
     return launch_kernel(cap ? kb : ka, dim3((unsigned)units), dim3(threads), smem, st, o.pdl, p, mapX,
-                         mapV, status, static_cast<const uint8_t*>(o.l2_hint), (uint32_t)o.l2_hint_bytes,
-                         o.next_maps[0], o.next_maps[1]);
+                         mapV, status, static_cast<const uint8_t*>(o.l2_hint), (uint32_t)o.l2_hint_bytes);
   } else {
     auto kernel = [] {
       if constexpr (UPB == 1) return k_input_transform_tma<M, MODE, CC, G, CPT, false>;
@@ -445,7 +438,7 @@ int input_tma_launch_u(const Params& p, const LaunchOpt& o, const CUtensorMap& m
     if (int rc = set_max_smem(once, o.device, kernel, smem)) return rc;
     return launch_kernel(kernel, dim3((unsigned)((units + UPB - 1) / UPB)), dim3(threads), smem, st, o.pdl,
                          p, mapX, mapV, status, static_cast<const uint8_t*>(o.l2_hint),
-                         (uint32_t)o.l2_hint_bytes, o.next_maps[0], o.next_maps[1]);
+                         (uint32_t)o.l2_hint_bytes);
   }
 }
 template <int M, int MODE, int CC, int G, int CPT>
