@@ -48,7 +48,8 @@ WINO_ST_READER(wino_trace_output, g_out_trace)
 #endif
 
 // Blocks per SM asked of the compiler.  One channel per thread: a full SM of threads (2048),
-// i.e. at most 32 registers each.  The output transform fits that without spilling.  The input
+// i.e. at most 32 registers each.  The F2 and F4 output transforms fit that without spilling
+// (F6 does not and is left alone).  The input
 // transform does not (it spills some sixty words), so it exists in two builds and the launcher
 // takes the 32-register one only where it turns a grid of slightly more than one wave into a
 // single wave: the 2048 blocks of a 256-channel, 1024-tile layer are then resident together,
@@ -276,7 +277,7 @@ k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_const
 }
 
 template <int M, int MODE, int KC, int G, int CPT>
-__global__ void __launch_bounds__((KC / CPT) * G, tma_min_blocks((KC / CPT) * G, CPT, true))
+__global__ void __launch_bounds__((KC / CPT) * G, tma_min_blocks((KC / CPT) * G, CPT, M <= 4))
 k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapM,
                        const __grid_constant__ CUtensorMap mapY, const float* __restrict__ bias,
                        float s_Y, int* __restrict__ status) {
@@ -417,7 +418,7 @@ int input_tma_launch_u(const Params& p, const LaunchOpt& o, const CUtensorMap& m
       2 * (size_t)UPB * G * ((((M + 2) * (M + 2) * CC) + 127) / 128 * 128) + 128 + 16 * UPB;
   constexpr int threads = (CC / CPT) * G;
   const int units = ((p.T + G - 1) / G) * (p.C / CC);
-  if constexpr (UPB == 1 && CPT == 1) {
+  if constexpr (UPB == 1 && CPT == 1 && M <= 4) {   // (F6 would spill an eighth of its work at 32 registers)
     // the 32-register build only where it saves a second wave
     static DeviceOnce once_a, once_b;
     auto ka = k_input_transform_tma<M, MODE, CC, G, CPT, false>;
