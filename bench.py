@@ -6,7 +6,7 @@
 One "step" is one forward pass of the layer (input transform, Hadamard-stage
 GEMMs, output transform, all quantizers) over one batch of the workload, with
 the transformed weights resident, as the paper treats them (Section 3.1: the
-weight transform is amortized across inferences); the weight transform is timed
+weight transform is done once and reused by every inference); it is timed
 separately and reported beside it.  The metric is effective direct-convolution-
 equivalent int8 TOPS: 2*N*H*W*K*C*9 operations per step over the measured time.
 
