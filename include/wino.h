@@ -216,7 +216,10 @@ int wino_calibrate_forward(wino_plan_t* plan, const int8_t* x_NHWC_dev,
  * (float)(bias/s_Y)); 1), float output fmaf((float)acc, (float)(s_x*s_w), bias).
  * x int8 [N][H][W][C], w int8 [K][3][3][C], y [N][Ho][Wo][K] with
  * Ho = (H-1)/stride + 1; C and K multiples of 4; device pointers 16-byte aligned.
- * Stateless: no plan, no workspace. */
+ * Stateless: no plan, no workspace.  Stride 1 without zero points on x and w, with
+ * C a multiple of 64, K a multiple of 32 (at most 2048) and y 32-byte aligned runs
+ * as an implicit GEMM on the tensor cores; everything else on the integer ALUs.
+ * The results are the same bits either way. */
 typedef struct {
   int32_t N, C, H, W, K, stride;
   wino_quant_t q_x, q_w, q_Y;
@@ -225,6 +228,11 @@ typedef struct {
 int wino_direct_conv_forward(const wino_direct_desc_t* desc, const int8_t* x_NHWC_dev,
                              const int8_t* w_KRSC_dev, const float* bias_K_dev, void* y_dev,
                              void* stream);
+/* Status of the direct convolutions on the current device, which have no plan to keep
+ * one in: synchronizes `stream`, returns WINO_OK, WINO_ERR_TIMEOUT (a bounded wait
+ * inside the tensor-core kernel expired; its output is undefined) or WINO_ERR_CUDA,
+ * and clears the word. */
+int wino_direct_last_status(void* stream);
 
 /* Synchronizes `stream` and returns the plan's device status word: WINO_OK, or
  * WINO_ERR_TIMEOUT if a bounded wait inside a kernel expired (the kernel then

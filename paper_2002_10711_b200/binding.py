@@ -27,7 +27,7 @@ EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
     "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward",
-    "wino_direct_conv_forward", "wino_last_status", "wino_debug_dump_stage",
+    "wino_direct_conv_forward", "wino_direct_last_status", "wino_last_status", "wino_debug_dump_stage",
     "wino_debug_forward_accumulators", "wino_debug_run_stages", "wino_debug_mma_probe",
     "wino_debug_wait_probe", "wino_debug_once_per_device", "wino_launch_count", "wino_destroy",
     "wino_strerror",
@@ -81,6 +81,7 @@ def _load() -> ct.CDLL:
     lib.wino_calibrate_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.wino_debug_run_stages.argtypes = [vp, i32, vp, vp, vp, vp, vp, vp]
     lib.wino_direct_conv_forward.argtypes = [ct.POINTER(DirectDescC), vp, vp, vp, vp, vp]
+    lib.wino_direct_last_status.argtypes = [vp]
     lib.wino_debug_mma_probe.argtypes = [vp, i32, vp]
     lib.wino_last_status.argtypes = [vp, vp]
     lib.wino_debug_dump_stage.argtypes = [vp, i32, vp, sz]
@@ -133,6 +134,11 @@ def _stream_handle(stream) -> ct.c_void_p:
 
 def debug_once_per_device(device: int) -> int:
     return _lib.wino_debug_once_per_device(device)
+
+
+def direct_last_status(stream=None) -> int:
+    """wino_direct_last_status: status word of the plan-less direct convolutions (read and cleared)."""
+    return int(_lib.wino_direct_last_status(_stream_handle(stream)))
 
 
 def direct_conv_forward(N, C, H, W, K, stride, q_x, q_w, q_Y, x_dev, w_dev, bias_dev, y_dev,

@@ -1,0 +1,284 @@
+// Direct int8 3x3 convolution, stride 1, as an implicit GEMM on the tensor cores
+// (the lossless "im2row" candidate of the paper's search space, Section 4, without ever
+// forming the im2row matrix).  For an output tile of 128 pixels and a block of BN output
+// channels,
+//     acc[pixel][k] = sum over the nine taps (a, b) and over c of x[n][h-1+a][w-1+b][c] * w[k][a][b][c],
+// i.e. nine GEMM K-slices per channel block.  The A operand of tap (a, b) is the input box
+// of the tile shifted by (a-1, b-1), fetched by one 4-D TMA load whose out-of-image part is
+// filled with zeros by the hardware (= the zero padding); the B operand is the tap's
+// [BN][channels] slice of the weights.  Both land in shared memory as K-major rows of 64 or
+// 128 channel bytes with the matching swizzle, `tcgen05.mma.kind::i8` accumulates all
+// 9 * C / 32 steps of an item in one tensor-memory accumulator, and sixteen epilogue warps
+// apply the output quantizer (or the float output) and write 32-byte row pieces.
+//
+//   warp 0    : TMA producer (one lane)
+//   warp 1    : tensor-memory owner; walks the MMA loop as a whole warp, one elected lane issues
+//   warps 2-17: epilogue; warp w reads TMEM lanes 32*(w%4) .. +31 and every fourth 32-column chunk
+//
+// Zero points on x or w, stride 2 and channel counts that are not multiples of 64 / 32 stay
+// on the ALU kernel (wino_direct.cu).
+#include "wino_launch.h"
+#include "wino_ptx.cuh"
+
+namespace wino {
+
+namespace {
+
+constexpr int kDtEpiWarps = 16;
+constexpr int kDtThreads = 64 + 32 * kDtEpiWarps;
+
+// K-major tile of 64-byte rows with the 64-byte swizzle: start / 16, 8-row group stride
+// 512 B, descriptor version 1, layout 4.
+__device__ __forceinline__ uint64_t desc_sw64(uint32_t smem_addr) {
+  return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | (1ull << 16) | (32ull << 32) | (1ull << 46) |
+         (4ull << 61);
+}
+
+__global__ void __launch_bounds__(kDtThreads, 1)
+k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
+                 const DirectTcArgs a, const float* __restrict__ bias, void* __restrict__ y,
+                 int* __restrict__ status) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  const uint32_t a_bytes = 128u * (uint32_t)a.cB, b_bytes = (uint32_t)a.BN * (uint32_t)a.cB;
+  const uint32_t stage_bytes = a_bytes + b_bytes;
+  const uint32_t s_bias = base + (uint32_t)a.stages * stage_bytes;   // K floats
+  const uint32_t bars = s_bias + (uint32_t)a.K * 4u;
+  const uint32_t bar_full = bars;                           // stages x 8 B
+  const uint32_t bar_empty = bar_full + 8u * a.stages;      // stages x 8 B
+  const uint32_t bar_acc_full = bar_empty + 8u * a.stages;  // 2 x 8 B
+  const uint32_t bar_acc_empty = bar_acc_full + 16u;        // 2 x 8 B
+  const uint32_t tmem_slot = bar_acc_empty + 16u;
+  const uint32_t abort_slot = tmem_slot + 4u;
+  uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
+  volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
+  volatile uint32_t* abort_p = reinterpret_cast<volatile uint32_t*>(gen + (abort_slot - base));
+  float* bias_tab = reinterpret_cast<float*>(gen + (s_bias - base));
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n_tiles = a.nW * a.nH * a.nI;
+  const int steps = 9 * a.KB;   // stages per item
+
+  griddep_launch();
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < a.stages; ++s) {
+      mbar_init(bar_full + 8u * s, 1);
+      mbar_init(bar_empty + 8u * s, 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(bar_acc_full + 8u * b, 1);
+      mbar_init(bar_acc_empty + 8u * b, kDtEpiWarps);
+    }
+    *abort_p = 0u;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    tma_prefetch_map(&mapX);
+    tma_prefetch_map(&mapW);
+  }
+  if (warp == 1) tmem_alloc(tmem_slot, (uint32_t)a.tmem_cols);
+  // bias in output-code units (or as it is, for the float output); the bias is a parameter of
+  // the layer, not an output of the preceding kernel
+  for (int k = threadIdx.x; k < a.K; k += blockDim.x) {
+    float b = 0.0f;
+    if (bias != nullptr)
+      b = a.out_dtype == 0 ? (float)((double)__ldg(bias + k) / (double)a.s_Y) : __ldg(bias + k);
+    bias_tab[k] = b;
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot_p;
+
+  if (warp == 0) {
+    if (lane == 0) {
+      int s = 0, issued = 0; uint32_t ph = 0;
+      griddep_wait();
+      for (int it = blockIdx.x; it < a.n_items; it += gridDim.x) {
+        const int nb = it / n_tiles, tile = it - nb * n_tiles;
+        const int tw = tile % a.nW, th = (tile / a.nW) % a.nH, ti = tile / (a.nW * a.nH);
+        bool ok = true;
+        for (int tap = 0; tap < 9 && ok; ++tap) {
+          const int ta = tap / 3, tb = tap - ta * 3;
+          for (int kb = 0; kb < a.KB; ++kb) {
+            if (issued >= a.stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
+            ++issued;
+            const uint32_t sa = base + (uint32_t)s * stage_bytes;
+            mbar_expect_tx(bar_full + 8u * s, stage_bytes);
+            // pixels outside the image (the padding ring, ragged tile edges, images past N)
+            // arrive as zeros
+            tma_load_4d(sa, &mapX, bar_full + 8u * s, kb * a.cB, tw * a.BW - 1 + tb, th * a.BH - 1 + ta,
+                        ti * a.BI);
+            tma_load_3d(sa + a_bytes, &mapW, bar_full + 8u * s, kb * a.cB, tap, nb * a.BN);
+            if (++s == a.stages) { s = 0; ph ^= 1u; }
+          }
+        }
+        if (!ok) { *abort_p = 1u; break; }
+      }
+    }
+  } else if (warp == 1) {
+    const bool leader = elect_one();
+    const uint32_t idesc = make_idesc_i8(128, a.BN);
+    const int ksteps = a.cB / 32;
+    int s = 0; uint32_t ph = 0;
+    int li = 0;
+    for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
+      const int buf = li & 1;
+      const uint32_t aph = (uint32_t)(li >> 1) & 1u;
+      bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8u * buf, aph ^ 1u, abort_p));
+      tc_fence_after();
+      const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride);
+      for (int st = 0; st < steps && ok; ++st) {
+        if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph, abort_p))) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = base + (uint32_t)s * stage_bytes;
+        const uint64_t da = a.cB == 128 ? make_desc_sw128(sa) : desc_sw64(sa);
+        const uint64_t db = a.cB == 128 ? make_desc_sw128(sa + a_bytes) : desc_sw64(sa + a_bytes);
+        if (leader) {
+          for (int k = 0; k < ksteps; ++k)
+            mma_i8(tacc, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (st | k) != 0 ? 1u : 0u);
+          mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
+        }
+        __syncwarp();
+        if (++s == a.stages) { s = 0; ph ^= 1u; }
+      }
+      if (!ok) { *abort_p = 1u; break; }
+      if (leader) mma_commit(bar_acc_full + 8u * buf);  // accumulator complete
+      __syncwarp();
+    }
+  } else {
+    const int quad = warp & 3;
+    const int sub = (warp - 2) >> 2;
+    const int r = quad * 32 + lane;
+    const int wi = r % a.BW, hi = (r / a.BW) % a.BH, ii = r / (a.BW * a.BH);
+    const float lo = a.lo_Y, hi_c = a.hi_Y;
+    griddep_wait();
+    int li = 0;
+    for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
+      const int nb = it / n_tiles, tile = it - nb * n_tiles;
+      const int tw = tile % a.nW, th = (tile / a.nW) % a.nH, ti = tile / (a.nW * a.nH);
+      const int n = ti * a.BI + ii, ho = th * a.BH + hi, wo = tw * a.BW + wi;
+      const bool valid = n < a.N && ho < a.H && wo < a.W;
+      const long pix = ((long)n * a.H + ho) * a.W + wo;
+      const int buf = li & 1;
+      const uint32_t aph = (uint32_t)(li >> 1) & 1u;
+      if (!__all_sync(0xffffffffu, mbar_wait(bar_acc_full + 8u * buf, aph, abort_p))) {
+        *abort_p = 1u;
+        break;
+      }
+      tc_fence_after();
+      const uint32_t tacc = tmem_base + (uint32_t)(buf * a.acc_stride) + ((uint32_t)(quad * 32) << 16);
+      for (int col = sub * 32; col < a.BN; col += 128) {
+        uint32_t acc[32];
+        tmem_ld32(tacc + (uint32_t)col, acc);
+        tmem_ld_wait();
+        if (!valid) continue;
+        const int k0 = nb * a.BN + col;
+        if (a.out_dtype == 0) {
+          uint32_t w[8];
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            uint32_t word = 0u;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+              const float yf = __fmaf_rn(__int2float_rn((int)acc[4 * q + e]), a.mult, bias_tab[k0 + 4 * q + e]);
+              const float rr = __fadd_rn(fminf(fmaxf(yf, lo), hi_c), kMagic);
+              word |= ((uint32_t)(magic_to_int(rr) + a.z_Y) & 0xFFu) << (8 * e);
+            }
+            w[q] = word;
+          }
+          uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(y) + pix * a.K + k0);
+          asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]),
+                       "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                       : "memory");
+        } else {
+          float4* dst = reinterpret_cast<float4*>(reinterpret_cast<float*>(y) + pix * a.K + k0);
+#pragma unroll
+          for (int q = 0; q < 8; ++q) {
+            float4 v;
+            v.x = __fmaf_rn(__int2float_rn((int)acc[4 * q + 0]), a.s_in, bias_tab[k0 + 4 * q + 0]);
+            v.y = __fmaf_rn(__int2float_rn((int)acc[4 * q + 1]), a.s_in, bias_tab[k0 + 4 * q + 1]);
+            v.z = __fmaf_rn(__int2float_rn((int)acc[4 * q + 2]), a.s_in, bias_tab[k0 + 4 * q + 2]);
+            v.w = __fmaf_rn(__int2float_rn((int)acc[4 * q + 3]), a.s_in, bias_tab[k0 + 4 * q + 3]);
+            dst[q] = v;
+          }
+        }
+      }
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty + 8u * buf);
+    }
+  }
+  __syncwarp();
+  tc_fence_before();
+  __syncthreads();
+  if (*abort_p != 0u && threadIdx.x == 0) atomicExch(status, -6);  // WINO_ERR_TIMEOUT
+  if (warp == 1) {
+    tc_fence_after();
+    tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
+  }
+}
+
+// One status word per device for the plan-less direct convolution.
+__device__ int g_direct_status;
+
+}  // namespace
+
+bool direct_tc_supported(int C, int K, int stride, int z_x, int z_w) {
+  return stride == 1 && z_x == 0 && z_w == 0 && C % 64 == 0 && K % 32 == 0 && K <= 2048;
+}
+
+DirectTcArgs direct_tc_geometry(int N, int C, int H, int W, int K, int num_sms) {
+  DirectTcArgs a = {};
+  a.N = N; a.C = C; a.H = H; a.W = W; a.K = K;
+  auto pow2_ceil = [](int v) { int p = 1; while (p < v) p *= 2; return p; };
+  a.BW = pow2_ceil(W) < 16 ? pow2_ceil(W) : 16;
+  a.BH = pow2_ceil(H) < 128 / a.BW ? pow2_ceil(H) : 128 / a.BW;
+  a.BI = 128 / (a.BW * a.BH);
+  a.nW = (W + a.BW - 1) / a.BW; a.nH = (H + a.BH - 1) / a.BH; a.nI = (N + a.BI - 1) / a.BI;
+  a.cB = C % 128 == 0 ? 128 : 64;
+  a.KB = C / a.cB;
+  a.BN = K % 256 == 0 ? 256 : K % 128 == 0 ? 128 : K % 64 == 0 ? 64 : 32;
+  const int tiles = a.nW * a.nH * a.nI;
+  // enough items for every SM, as long as the blocks stay at least 64 channels wide
+  while (a.BN > 64 && tiles * (K / a.BN) < (num_sms * 4) / 5) a.BN /= 2;
+  a.n_nblk = K / a.BN;
+  a.n_items = tiles * a.n_nblk;
+  const size_t stage = (size_t)128 * a.cB + (size_t)a.BN * a.cB;
+  a.stages = (int)((192 * 1024) / stage);
+  if (a.stages > 8) a.stages = 8;
+  int acc_stride = 32;
+  while (acc_stride < a.BN) acc_stride *= 2;
+  a.acc_stride = acc_stride;
+  a.tmem_cols = 2 * acc_stride;
+  return a;
+}
+
+int* direct_tc_status_word(int device) {
+  static std::mutex mu;
+  static int* addr[64];
+  std::lock_guard<std::mutex> lock(mu);
+  const int d = device >= 0 && device < 64 ? device : 0;
+  if (addr[d] == nullptr) {
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_direct_status) != cudaSuccess) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    addr[d] = static_cast<int*>(p);
+  }
+  return addr[d];
+}
+
+int launch_direct_conv_tc(const DirectTcArgs& a, int device, int num_sms, const CUtensorMap& mapX,
+                          const CUtensorMap& mapW, const float* bias, void* y, cudaStream_t st) {
+  int* status = direct_tc_status_word(device);
+  if (status == nullptr) return -5;
+  const size_t stage = (size_t)128 * a.cB + (size_t)a.BN * a.cB;
+  const size_t smem = 1024 + (size_t)a.stages * stage + (size_t)a.K * 4 + 16 * (size_t)a.stages + 64;
+  static DeviceOnce once;
+  if (int rc = set_max_smem(once, device, k_direct_conv_tc, 227 * 1024)) return rc;
+  const int grid = a.n_items < num_sms ? a.n_items : num_sms;
+  return launch_kernel(k_direct_conv_tc, dim3((unsigned)grid), dim3(kDtThreads), smem, st, true, mapX, mapW,
+                       a, bias, y, status);
+}
+
+}  // namespace wino

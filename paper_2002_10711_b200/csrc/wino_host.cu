@@ -605,12 +605,51 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
   if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
   const double s_in = (double)d->q_x.scale * (double)d->q_w.scale;
+  if (direct_tc_supported(d->C, d->K, d->stride, d->q_x.zero_point, d->q_w.zero_point) &&
+      (reinterpret_cast<uintptr_t>(y) & 31u) == 0) {
+    // implicit GEMM on the tensor cores: x as [N][H][W][C] boxes of one output tile, w as
+    // [K][9][C] slices of one tap
+    int dev = 0, sms = 148;
+    if (cudaGetDevice(&dev) != cudaSuccess) return WINO_ERR_CUDA;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
+      sms = 148;
+    DirectTcArgs a = direct_tc_geometry(d->N, d->C, d->H, d->W, d->K, sms);
+    a.mult = (float)(s_in / (double)d->q_Y.scale);
+    a.s_in = (float)s_in;
+    a.s_Y = d->q_Y.scale;
+    a.lo_Y = (float)(d->q_Y.qmin - d->q_Y.zero_point);
+    a.hi_Y = (float)(d->q_Y.qmax - d->q_Y.zero_point);
+    a.z_Y = d->q_Y.zero_point;
+    a.out_dtype = d->out_dtype;
+    const CUtensorMapSwizzle swz = a.cB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    CUtensorMap mapX, mapW;
+    const uint64_t xd[4] = {(uint64_t)d->C, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)d->N};
+    const uint32_t xb[4] = {(uint32_t)a.cB, (uint32_t)a.BW, (uint32_t)a.BH, (uint32_t)a.BI};
+    const uint64_t wd[3] = {(uint64_t)d->C, 9, (uint64_t)d->K};
+    const uint32_t wb[3] = {(uint32_t)a.cB, 1, (uint32_t)a.BN};
+    if (encode_tiled(&mapX, x, 4, xd, xb, swz) != WINO_OK || encode_tiled(&mapW, w, 3, wd, wb, swz) != WINO_OK)
+      return WINO_ERR_CUDA;
+    return launch_direct_conv_tc(a, dev, sms, mapX, mapW, bias, y, (cudaStream_t)stream) == 0
+               ? WINO_OK : WINO_ERR_CUDA;
+  }
   return launch_direct_conv(d->N, d->C, d->H, d->W, d->K, d->stride, d->q_x.zero_point,
                             d->q_w.zero_point, d->q_Y.zero_point,
                             (float)(s_in / (double)d->q_Y.scale), (float)s_in, d->q_Y.scale,
                             (float)(d->q_Y.qmin - d->q_Y.zero_point),
                             (float)(d->q_Y.qmax - d->q_Y.zero_point), d->out_dtype, x, w, bias, y,
                             (cudaStream_t)stream);
+}
+
+int wino_direct_last_status(void* stream) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return WINO_ERR_CUDA;
+  int* word = direct_tc_status_word(dev);
+  if (word == nullptr) return WINO_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return WINO_ERR_CUDA;
+  int v = 0;
+  if (cudaMemcpy(&v, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) return WINO_ERR_CUDA;
+  if (v != 0 && cudaMemset(word, 0, sizeof(int)) != cudaSuccess) return WINO_ERR_CUDA;
+  return v;
 }
 
 int wino_debug_mma_probe(wino_plan_t* pl, int iters, void* stream) {

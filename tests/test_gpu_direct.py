@@ -23,8 +23,12 @@ def _run(N, C, H, W, K, stride, q_x, q_w, q_Y, x_q, w_q, bias, out_dtype=0):
     return y.cpu().numpy()
 
 
+# the second row of shapes runs on the tensor cores at stride 1 without zero points (C % 64 == 0,
+# K % 32 == 0): ragged tiles, tiles spanning several images, 64- and 128-byte channel blocks
 @pytest.mark.parametrize("shape", [(2, 16, 9, 7, 8), (1, 64, 32, 32, 128), (3, 4, 1, 1, 4), (2, 128, 16, 16, 256),
-                                   (1, 20, 6, 11, 12)])
+                                   (1, 20, 6, 11, 12),
+                                   (3, 128, 8, 8, 64), (5, 64, 4, 4, 96), (1, 256, 5, 19, 32), (2, 192, 1, 1, 64),
+                                   (1, 512, 4, 4, 512), (2, 64, 9, 7, 32)])
 @pytest.mark.parametrize("stride", [1, 2])
 @pytest.mark.parametrize("variant", ["plain", "relu_bias", "zero_points"])
 def test_direct_conv_matches_oracle(shape, stride, variant):
@@ -49,6 +53,8 @@ def test_direct_conv_matches_oracle(shape, stride, variant):
                q_Y, x_q, w_q, bias)
     assert got.shape == want.shape and (got == want).all()
     assert want.size < 100 or len(np.unique(want)) > 3
+    from paper_2002_10711_b200 import binding
+    assert binding.direct_last_status() == 0
 
 
 def test_direct_conv_float_output():
@@ -62,6 +68,35 @@ def test_direct_conv_float_output():
     want = acc.astype(np.float32).astype(np.float64) * np.float64(s_in) + bias.astype(np.float64)
     got = _run(N, C, H, W, K, 2, Quant(scale=s_x), Quant(scale=float(s_w)), Quant(), x_q, w_q, bias, out_dtype=1)
     assert float(np.abs(got - want).max()) <= 1e-4 * float(np.abs(want).max())
+
+
+def test_direct_conv_float_output_tensor_core_path():
+    N, C, H, W, K = 2, 64, 10, 9, 32
+    x_q = wi.halfnormal_codes(5200, 1, (N, H, W, C))
+    w_q, s_w = wi.gaussian_weight_codes(5200, 2, (K, 3, 3, C), 0.05)
+    bias = wi.bias_values(5200, 3, K, 0.5)
+    s_x = float(np.float32(1 / 32))
+    acc = oracle.direct_conv_i32(x_q, w_q, stride=1)
+    s_in = np.float32(s_x * float(s_w))
+    want = acc.astype(np.float32).astype(np.float64) * np.float64(s_in) + bias.astype(np.float64)
+    got = _run(N, C, H, W, K, 1, Quant(scale=s_x), Quant(scale=float(s_w)), Quant(), x_q, w_q, bias, out_dtype=1)
+    assert float(np.abs(got - want).max()) <= 1e-4 * float(np.abs(want).max())
+
+
+def test_direct_conv_resnet_layer_shapes_at_batch():
+    # the layer shapes of the ResNet-18 body at a batch that fills the GPU several times over
+    for (N, C, H, W, K) in [(32, 64, 32, 32, 64), (32, 256, 8, 8, 256)]:
+        x_q = wi.halfnormal_codes(5300 + C, 1, (N, H, W, C))
+        w_q, s_w = wi.gaussian_weight_codes(5300 + K, 2, (K, 3, 3, C), 0.05)
+        s_x = float(np.float32(1 / 32))
+        acc = oracle.direct_conv_i32(x_q, w_q, stride=1)
+        s_in = s_x * float(s_w)
+        q_Y = Quant(qmin=0)
+        q_Y.scale = float(np.float32(float(np.abs(acc).max()) * s_in / 127.0))
+        bias = wi.bias_values(5300, 3, K, 0.5)
+        want = oracle.requantize_acc(acc, s_in, q_Y, bias)
+        got = _run(N, C, H, W, K, 1, Quant(scale=s_x), Quant(scale=float(s_w)), q_Y, x_q, w_q, bias)
+        assert (got == want).all()
 
 
 def test_direct_conv_argument_checks():
