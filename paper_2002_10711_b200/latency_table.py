@@ -4,11 +4,10 @@ This is the lookup table a latency-aware search over convolution algorithms
 needs (paper: Section 4, "each candidate operation comes with its respective
 latency"); the paper filled it on Arm cores.
 
-    python -m paper_2002_10711_b200.latency_table [--batch 256]
+    python -m paper_2002_10711_b200.latency_table [--batch 256] [--channels 256]
 
-The direct convolution here is the library's integer-dot-product kernel on the
-ALUs (it exists for the strided layers); it is not a tensor-core implicit GEMM, so
-its column is an upper bound on what a tuned direct convolution would take.
+The direct convolution is the library's implicit GEMM on the tensor cores (stride 1,
+channel counts that are multiples of 64 / 32; other layers run on the integer ALUs).
 
 Prints one JSON object per shape.  Steady-state time per call: the call is
 captured in a CUDA graph on rotating buffers and timed with CUDA events.
@@ -79,8 +78,11 @@ def layer_latencies(N, C, H, W, K, device="cuda:0", sets=8):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--batch", type=int, default=256)
+    ap.add_argument("--channels", type=int, default=0, help="only the layer shape of this width")
     args = ap.parse_args()
     for C, S in RESNET18_CIFAR:
+        if args.channels and C != args.channels:
+            continue
         lat = layer_latencies(args.batch, C, S, S, C)
         best = min((v, k) for k, v in lat.items() if v is not None)[1]
         print(json.dumps({"N": args.batch, "C": C, "K": C, "H": S, "W": S,
