@@ -99,6 +99,34 @@ def test_direct_conv_resnet_layer_shapes_at_batch():
         assert (got == want).all()
 
 
+def test_direct_conv_tensor_core_path_writes_nothing_outside_y():
+    # ragged tiles (W = 19 > 16, H = 5 < 8) and a tile that spans images past N: the output sits
+    # between guard bands that must keep their pattern
+    import torch
+    from paper_2002_10711_b200 import binding
+    for (N, C, H, W, K) in [(1, 64, 5, 19, 32), (3, 128, 8, 8, 64), (5, 64, 4, 4, 96)]:
+        x_q = wi.halfnormal_codes(5400 + C, 1, (N, H, W, C))
+        w_q, s_w = wi.gaussian_weight_codes(5400 + K, 2, (K, 3, 3, C), 0.05)
+        s_x = float(np.float32(1 / 32))
+        acc = oracle.direct_conv_i32(x_q, w_q, stride=1)
+        s_in = s_x * float(s_w)
+        q_Y = Quant(scale=float(np.float32(float(np.abs(acc).max()) * s_in / 127.0)))
+        want = oracle.requantize_acc(acc, s_in, q_Y, None)
+        guard = 4096
+        nbytes = N * H * W * K
+        arena = torch.full((guard + nbytes + guard,), 0x5A, dtype=torch.uint8, device="cuda")
+        y = arena[guard:guard + nbytes].view(torch.int8).view(N, H, W, K)
+        assert y.data_ptr() % 32 == 0
+        x = torch.from_numpy(x_q).cuda()
+        w = torch.from_numpy(w_q).cuda()
+        binding.direct_conv_forward(N, C, H, W, K, 1, Quant(scale=s_x), Quant(scale=float(s_w)), q_Y, x, w, None, y)
+        torch.cuda.synchronize()
+        assert binding.direct_last_status() == 0
+        a = arena.cpu().numpy()
+        assert (a[:guard] == 0x5A).all() and (a[guard + nbytes:] == 0x5A).all()
+        assert (a[guard:guard + nbytes].view(np.int8).reshape(N, H, W, K) == want).all()
+
+
 def test_direct_conv_argument_checks():
     from paper_2002_10711_b200 import binding
     q = Quant()
