@@ -1,8 +1,8 @@
-// Direct int8 3x3 convolution, stride 1, as an implicit GEMM on the tensor cores
+// Direct int8 3x3 convolution, stride 1 or 2, as an implicit GEMM on the tensor cores
 // (the lossless "im2row" candidate of the paper's search space, Section 4, without ever
 // forming the im2row matrix).  For an output tile of 128 pixels and a block of BN output
 // channels,
-//     acc[pixel][k] = sum over the nine taps (a, b) and over c of x[n][h-1+a][w-1+b][c] * w[k][a][b][c],
+//     acc[pixel][k] = sum over the nine taps (a, b) and over c of x[n][s*h-1+a][s*w-1+b][c] * w[k][a][b][c],
 // i.e. nine GEMM K-slices per channel block.  The A operand of tap (a, b) is the input box
 // of the tile shifted by (a-1, b-1), fetched by one 4-D TMA load whose out-of-image part is
 // filled with zeros by the hardware (= the zero padding); the B operand is the tap's
@@ -15,8 +15,10 @@
 //   warp 1    : tensor-memory owner; walks the MMA loop as a whole warp, one elected lane issues
 //   warps 2-17: epilogue; warp w reads TMEM lanes 32*(w%4) .. +31 and every fourth 32-column chunk
 //
-// Zero points on x or w, stride 2 and channel counts that are not multiples of 64 / 32 stay
-// on the ALU kernel (wino_direct.cu).
+// For stride 2 (even H and W) the input is addressed as [N][H/2][2][W/2][2*C]: a tap then reads
+// one row parity and one column parity, again a dense box.
+// Zero points on x or w, odd sizes at stride 2 and channel counts that are not multiples of
+// 64 / 32 stay on the ALU kernel (wino_direct.cu).
 #include "wino_launch.h"
 #include "wino_ptx.cuh"
 
@@ -105,8 +107,16 @@ k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant
             mbar_expect_tx(bar_full + 8u * s, stage_bytes);
             // pixels outside the image (the padding ring, ragged tile edges, images past N)
             // arrive as zeros
-            tma_load_4d(sa, &mapX, bar_full + 8u * s, kb * a.cB, tw * a.BW - 1 + tb, th * a.BH - 1 + ta,
-                        ti * a.BI);
+            if (a.stride == 1) {
+              tma_load_4d(sa, &mapX, bar_full + 8u * s, kb * a.cB, tw * a.BW - 1 + tb, th * a.BH - 1 + ta,
+                          ti * a.BI);
+            } else {
+              // input row 2*ho - 1 + ta: (half-row ho - 1, parity 1), (ho, 0), (ho, 1) for ta = 0, 1, 2
+              const int pcol = tb == 1 ? 0 : 1, dw = tb == 0 ? -1 : 0;
+              const int prow = ta == 1 ? 0 : 1, dh = ta == 0 ? -1 : 0;
+              tma_load_5d(sa, &mapX, bar_full + 8u * s, pcol * a.C + kb * a.cB, tw * a.BW + dw, prow,
+                          th * a.BH + dh, ti * a.BI);
+            }
             tma_load_3d(sa + a_bytes, &mapW, bar_full + 8u * s, kb * a.cB, tap, nb * a.BN);
             if (++s == a.stages) { s = 0; ph ^= 1u; }
           }
@@ -222,13 +232,15 @@ __device__ int g_direct_status;
 
 }  // namespace
 
-bool direct_tc_supported(int C, int K, int stride, int z_x, int z_w) {
-  return stride == 1 && z_x == 0 && z_w == 0 && C % 64 == 0 && K % 32 == 0 && K <= 2048;
+bool direct_tc_supported(int C, int K, int H, int W, int stride, int z_x, int z_w) {
+  if (z_x != 0 || z_w != 0 || C % 64 != 0 || K % 32 != 0 || K > 2048) return false;
+  return stride == 1 || (stride == 2 && H % 2 == 0 && W % 2 == 0);
 }
 
-DirectTcArgs direct_tc_geometry(int N, int C, int H, int W, int K, int num_sms) {
+DirectTcArgs direct_tc_geometry(int N, int C, int H_in, int W_in, int K, int stride, int num_sms) {
   DirectTcArgs a = {};
-  a.N = N; a.C = C; a.H = H; a.W = W; a.K = K;
+  const int H = (H_in - 1) / stride + 1, W = (W_in - 1) / stride + 1;   // output size
+  a.N = N; a.C = C; a.H = H; a.W = W; a.K = K; a.stride = stride;
   auto pow2_ceil = [](int v) { int p = 1; while (p < v) p *= 2; return p; };
   a.BW = pow2_ceil(W) < 16 ? pow2_ceil(W) : 16;
   a.BH = pow2_ceil(H) < 128 / a.BW ? pow2_ceil(H) : 128 / a.BW;

@@ -166,8 +166,8 @@ int encode_tiled(CUtensorMap* map, const void* base, int rank, const uint64_t* d
                  const uint32_t* box, CUtensorMapSwizzle swz) {
   EncodeTiledFn fn = get_encode_fn();
   if (fn == nullptr) return WINO_ERR_CUDA;
-  cuuint64_t d[4], strides[3];
-  cuuint32_t b[4], estr[4] = {1, 1, 1, 1};
+  cuuint64_t d[5], strides[4];
+  cuuint32_t b[5], estr[5] = {1, 1, 1, 1, 1};
   uint64_t stride = 1;
   for (int i = 0; i < rank; ++i) {
     d[i] = dims[i];
@@ -605,7 +605,7 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
   if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
   const double s_in = (double)d->q_x.scale * (double)d->q_w.scale;
-  if (direct_tc_supported(d->C, d->K, d->stride, d->q_x.zero_point, d->q_w.zero_point) &&
+  if (direct_tc_supported(d->C, d->K, d->H, d->W, d->stride, d->q_x.zero_point, d->q_w.zero_point) &&
       (reinterpret_cast<uintptr_t>(y) & 31u) == 0) {
     // implicit GEMM on the tensor cores: x as [N][H][W][C] boxes of one output tile, w as
     // [K][9][C] slices of one tap
@@ -613,7 +613,7 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
     if (cudaGetDevice(&dev) != cudaSuccess) return WINO_ERR_CUDA;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1)
       sms = 148;
-    DirectTcArgs a = direct_tc_geometry(d->N, d->C, d->H, d->W, d->K, sms);
+    DirectTcArgs a = direct_tc_geometry(d->N, d->C, d->H, d->W, d->K, d->stride, sms);
     a.mult = (float)(s_in / (double)d->q_Y.scale);
     a.s_in = (float)s_in;
     a.s_Y = d->q_Y.scale;
@@ -623,12 +623,23 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
     a.out_dtype = d->out_dtype;
     const CUtensorMapSwizzle swz = a.cB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
     CUtensorMap mapX, mapW;
-    const uint64_t xd[4] = {(uint64_t)d->C, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)d->N};
-    const uint32_t xb[4] = {(uint32_t)a.cB, (uint32_t)a.BW, (uint32_t)a.BH, (uint32_t)a.BI};
+    int rcx;
+    if (d->stride == 1) {
+      const uint64_t xd[4] = {(uint64_t)d->C, (uint64_t)d->W, (uint64_t)d->H, (uint64_t)d->N};
+      const uint32_t xb[4] = {(uint32_t)a.cB, (uint32_t)a.BW, (uint32_t)a.BH, (uint32_t)a.BI};
+      rcx = encode_tiled(&mapX, x, 4, xd, xb, swz);
+    } else {
+      // stride 2 (H and W even): x as [N][H/2][2][W/2][2*C], so that the pixels an output tile
+      // needs for one tap (every other row and column) are a dense box with the row and column
+      // parities as coordinates
+      const uint64_t xd[5] = {(uint64_t)(2 * d->C), (uint64_t)(d->W / 2), 2, (uint64_t)(d->H / 2),
+                              (uint64_t)d->N};
+      const uint32_t xb[5] = {(uint32_t)a.cB, (uint32_t)a.BW, 1, (uint32_t)a.BH, (uint32_t)a.BI};
+      rcx = encode_tiled(&mapX, x, 5, xd, xb, swz);
+    }
     const uint64_t wd[3] = {(uint64_t)d->C, 9, (uint64_t)d->K};
     const uint32_t wb[3] = {(uint32_t)a.cB, 1, (uint32_t)a.BN};
-    if (encode_tiled(&mapX, x, 4, xd, xb, swz) != WINO_OK || encode_tiled(&mapW, w, 3, wd, wb, swz) != WINO_OK)
-      return WINO_ERR_CUDA;
+    if (rcx != WINO_OK || encode_tiled(&mapW, w, 3, wd, wb, swz) != WINO_OK) return WINO_ERR_CUDA;
     return launch_direct_conv_tc(a, dev, sms, mapX, mapW, bias, y, (cudaStream_t)stream) == 0
                ? WINO_OK : WINO_ERR_CUDA;
   }

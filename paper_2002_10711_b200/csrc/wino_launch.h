@@ -129,9 +129,11 @@ int launch_fused_f2(const Params& p, const LaunchOpt& o, const CUtensorMap& mapU
                     cudaStream_t st);
 
 // Direct int8 3x3 convolution (stride 1 or 2) on the ALUs.
-// Tensor-core direct convolution (stride 1, no zero points on x and w, C % 64 == 0, K % 32 == 0).
+// Tensor-core direct convolution (no zero points on x and w, C % 64 == 0, K % 32 == 0; stride 2
+// with even H and W).
 struct DirectTcArgs {
-  int N, C, H, W, K;
+  int N, C, H, W, K;       // H, W: output height and width
+  int stride;
   int BW, BH, BI;          // output tile: BW x BH pixels of BI images, BW * BH * BI = 128
   int nW, nH, nI;          // tiles along width, height, batch
   int BN, n_nblk;          // output-channel block and their number
@@ -141,8 +143,8 @@ struct DirectTcArgs {
   float mult, s_in, s_Y, lo_Y, hi_Y;
   int z_Y, out_dtype;
 };
-bool direct_tc_supported(int C, int K, int stride, int z_x, int z_w);
-DirectTcArgs direct_tc_geometry(int N, int C, int H, int W, int K, int num_sms);
+bool direct_tc_supported(int C, int K, int H, int W, int stride, int z_x, int z_w);
+DirectTcArgs direct_tc_geometry(int N, int C, int H, int W, int K, int stride, int num_sms);
 int* direct_tc_status_word(int device);
 int launch_direct_conv_tc(const DirectTcArgs& a, int device, int num_sms, const CUtensorMap& mapX,
                           const CUtensorMap& mapW, const float* bias, void* y, cudaStream_t st);
