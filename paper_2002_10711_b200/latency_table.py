@@ -4,7 +4,7 @@ This is the lookup table a latency-aware search over convolution algorithms
 needs (paper: Section 4, "each candidate operation comes with its respective
 latency"); the paper filled it on Arm cores.
 
-    python -m paper_2002_10711_b200.latency_table [--batch 256] [--channels 256]
+    python -m paper_2002_10711_b200.latency_table [--batch 256] [--channels 256] [--strided]
 
 The direct convolution is the library's implicit GEMM on the tensor cores (stride 1,
 channel counts that are multiples of 64 / 32; other layers run on the integer ALUs).
@@ -75,11 +75,32 @@ def layer_latencies(N, C, H, W, K, device="cuda:0", sets=8):
     return out
 
 
+def strided_latency(N, C, H, W, K, device="cuda:0", sets=8):
+    """Microseconds per call of the stride-2 direct convolution C -> K on an H x W input."""
+    dev = torch.device(device)
+    gen = torch.Generator(device="cpu").manual_seed(2)
+    xs = [torch.randint(0, 127, (N, H, W, C), dtype=torch.int8, generator=gen).to(dev) for _ in range(sets)]
+    w = torch.randint(-127, 127, (K, 3, 3, C), dtype=torch.int8, generator=gen).to(dev)
+    ys = [torch.empty((N, (H - 1) // 2 + 1, (W - 1) // 2 + 1, K), dtype=torch.int8, device=dev)
+          for _ in range(sets)]
+    q = dict(scale=0.05)
+    t = _time_graph(lambda i: binding.direct_conv_forward(
+        N, C, H, W, K, 2, q, q, dict(scale=4.0), xs[i % sets], w, None, ys[i % sets]))
+    assert binding.direct_last_status() == 0
+    return t
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--batch", type=int, default=256)
     ap.add_argument("--channels", type=int, default=0, help="only the layer shape of this width")
+    ap.add_argument("--strided", action="store_true",
+                    help="also the network's three stride-2 layers (direct convolution only)")
     args = ap.parse_args()
+    if args.strided:
+        for (C, S), (K, _) in zip(RESNET18_CIFAR[:-1], RESNET18_CIFAR[1:]):
+            print(json.dumps({"N": args.batch, "C": C, "K": K, "H": S, "W": S, "stride": 2,
+                              "us": {"direct": round(strided_latency(args.batch, C, S, S, K), 1)}}), flush=True)
     for C, S in RESNET18_CIFAR:
         if args.channels and C != args.channels:
             continue
