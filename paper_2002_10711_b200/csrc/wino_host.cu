@@ -476,11 +476,15 @@ int wino_plan(const wino_desc_t* desc, wino_plan_t** out) {
   p.out_dtype = d.out_dtype;
   pl->std_mats = d.m == 2 ? is_std<2>(p.BT, p.AT) : d.m == 4 ? is_std<4>(p.BT, p.AT)
                                                                : is_std<6>(p.BT, p.AT);
-  // Automatic choice, by measurement on B200: the fused F2 kernel where it applies,
-  // else the staged tcgen05 path, else the staged dp4a path.  The warp-shuffle
-  // small-channel kernel stays selectable (wino_plan_force_path) but the staged
-  // paths were faster on every layer size tried, tiny batches included.
+  // Automatic choice, by measurement on B200: the fused F2 kernel where it applies; for
+  // layers of at most 16 channels in and out the staged path with integer dot products on the
+  // ALUs (a 16-wide GEMM leaves the tensor-core pipeline mostly empty: 54 against 73 us at
+  // 16 channels, 32x32, batch 256, F2); else the staged tcgen05 path, else the staged dp4a
+  // path.  The warp-shuffle small-channel kernel stays selectable (wino_plan_force_path) but
+  // a staged path was faster on every layer size tried, tiny batches included.
   if (path_supported(pl, WINO_PATH_FUSED_F2)) pl->path = WINO_PATH_FUSED_F2;
+  else if (d.C <= 16 && d.K <= 16 && path_supported(pl, WINO_PATH_STAGED_DP4A))
+    pl->path = WINO_PATH_STAGED_DP4A;
   else if (path_supported(pl, WINO_PATH_STAGED_TC)) pl->path = WINO_PATH_STAGED_TC;
   else if (path_supported(pl, WINO_PATH_STAGED_DP4A)) pl->path = WINO_PATH_STAGED_DP4A;
   else { delete pl; return WINO_ERR_UNSUPPORTED; }

@@ -50,7 +50,8 @@ def test_sizes_and_paths():
     assert p.T == 2 * 2 * 2
     assert p.workspace_bytes >= 36 * p.T * 64 * 2
     assert p.path == binding.PATH_STAGED_TC
-    assert _plan(C=16, K=16).path == binding.PATH_STAGED_TC
+    assert _plan(C=16, K=16).path == binding.PATH_STAGED_DP4A     # at most 16 channels: integer dot products
+    assert _plan(C=32, K=16).path == binding.PATH_STAGED_TC
     assert _plan(C=20, K=24).path == binding.PATH_STAGED_DP4A
     p = _plan(C=20, K=24)
     p.force_path(binding.PATH_SMALLC)
