@@ -95,6 +95,7 @@ struct GemmTcArgs {
   int out_mode;
   int MB;          // m-blocks (128 tiles each) per work item, sharing one U_q tile
   int n_mblk, n_nblk, n_items;   // n_mblk counts groups of MB m-blocks
+  int wide_store;  // 1: the output rows are 32-byte aligned (one 256-bit store per row piece)
 };
 
 template <bool SMALL>
@@ -107,7 +108,8 @@ __device__ __forceinline__ float acc_to_float(uint32_t v) {
 // are inside K (no per-element guards).  STATS: track max |M| for calibration.
 template <bool SMALL, bool FULL, bool STATS>
 __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (&r)[32], int k0,
-                                               long o, int out_mode, void* out, float& vmax) {
+                                               long o, int out_mode, void* out, float& vmax,
+                                               bool wide_store) {
   if constexpr (STATS) {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -136,14 +138,14 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
                                   p.mult_M, lo_m, hi_m);
     }
     uint4* dst = reinterpret_cast<uint4*>(reinterpret_cast<int8_t*>(out) + o);
-    if constexpr (FULL) {
+    if (FULL && wide_store) {
       // the whole 32-byte sector of this row in one request
       asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst), "r"(w[0]),
                    "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
                    : "memory");
     } else {
-      if (k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
-      if (k0 + 16 < p.K) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
+      if (FULL || k0 < p.K) dst[0] = make_uint4(w[0], w[1], w[2], w[3]);
+      if (FULL || k0 + 16 < p.K) dst[1] = make_uint4(w[4], w[5], w[6], w[7]);
     }
   }
 }
@@ -186,7 +188,7 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
       if (tau >= p.T) continue;
       const int k0 = nb * a.BN + kcol;
       const long o = ((long)xi * p.T + tau) * p.K + k0;
-      epilogue_chunk<SMALL, FULL, STATS>(p, r0, k0, o, a.out_mode, out, vmax);
+      epilogue_chunk<SMALL, FULL, STATS>(p, r0, k0, o, a.out_mode, out, vmax, a.wide_store != 0);
     }
     tc_fence_before();
     __syncwarp();
@@ -412,6 +414,7 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
   a.n_mblk = ((p.T + kBM - 1) / kBM + g.MB - 1) / g.MB;
   a.n_nblk = (p.K + g.BN - 1) / g.BN;
   a.n_items = p.t * p.t * a.n_mblk * a.n_nblk;
+  a.wide_store = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
   return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,
                        mapV, mapU, a, out, absmaxM, status);
 }
