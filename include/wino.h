@@ -215,7 +215,9 @@ int wino_calibrate_forward(wino_plan_t* plan, const int8_t* x_NHWC_dev,
  * is the real value zero); int8 output Q(fmaf((float)acc, (float)(s_x*s_w/s_Y),
  * (float)(bias/s_Y)); 1), float output fmaf((float)acc, (float)(s_x*s_w), bias).
  * x int8 [N][H][W][C], w int8 [K][3][3][C], y [N][Ho][Wo][K] with
- * Ho = (H-1)/stride + 1; C and K multiples of 4; device pointers 16-byte aligned.
+ * Ho = (H-1)/stride + 1; any C and K (a layer whose C or K is not a multiple of 4,
+ * such as a three-channel first layer, runs on a simple byte-wise kernel); device
+ * pointers 16-byte aligned.
  * Stateless: no plan, no workspace.  Without zero points on x and w, with C a
  * multiple of 64, K a multiple of 32 (at most 2048), y 32-byte aligned and, at
  * stride 2, even H and W, the layer runs as an implicit GEMM on the tensor cores;

@@ -88,6 +88,45 @@ k_direct_conv(const DirectParams p, const int8_t* __restrict__ x, const int8_t* 
   }
 }
 
+// Any channel counts (the network's three-channel first layer, Section 5.1): thread =
+// (output pixel, output channel), byte loads.  Small layers only; nothing here is tuned.
+__global__ void __launch_bounds__(128)
+k_direct_conv_bytes(const DirectParams p, const int8_t* __restrict__ x, const int8_t* __restrict__ w,
+                    const float* __restrict__ bias, void* __restrict__ y) {
+  const long npix = (long)p.N * p.Ho * p.Wo;
+  const long idx = blockIdx.x * (long)blockDim.x + threadIdx.x;
+  griddep_launch();
+  griddep_wait();
+  if (idx >= npix * p.K) return;
+  const int k = (int)(idx % p.K);             // consecutive lanes: consecutive output channels
+  long pix = idx / p.K;
+  const int wo = (int)(pix % p.Wo); pix /= p.Wo;
+  const int ho = (int)(pix % p.Ho);
+  const int n = (int)(pix / p.Ho);
+  int acc = 0;
+  for (int a = 0; a < 3; ++a) {
+    const int h = ho * p.stride - 1 + a;
+    if (h < 0 || h >= p.H) continue;
+    for (int b = 0; b < 3; ++b) {
+      const int wv = wo * p.stride - 1 + b;
+      if (wv < 0 || wv >= p.W) continue;      // padding is the real value zero
+      const int8_t* xp = x + (((long)n * p.H + h) * p.W + wv) * p.C;
+      const int8_t* wp = w + (((long)k * 3 + a) * 3 + b) * p.C;
+      for (int c = 0; c < p.C; ++c) acc += ((int)__ldg(xp + c) - p.z_x) * ((int)__ldg(wp + c) - p.z_w);
+    }
+  }
+  const long o = (((long)n * p.Ho + ho) * p.Wo + wo) * p.K + k;
+  if (p.out_dtype == 0) {
+    const float b = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)p.s_Y) : 0.0f;
+    const float yf = __fmaf_rn(__int2float_rn(acc), p.mult, b);
+    const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
+    reinterpret_cast<int8_t*>(y)[o] = (int8_t)(magic_to_int(r) + p.z_Y);
+  } else {
+    const float b = bias != nullptr ? __ldg(bias + k) : 0.0f;
+    reinterpret_cast<float*>(y)[o] = __fmaf_rn(__int2float_rn(acc), p.s_in, b);
+  }
+}
+
 int launch_direct_conv(int N, int C, int H, int W, int K, int stride, int z_x, int z_w, int z_Y,
                        float mult, float s_in, float s_Y, float lo_Y, float hi_Y, int out_dtype,
                        const int8_t* x, const int8_t* w, const float* bias, void* y,
@@ -99,6 +138,12 @@ int launch_direct_conv(int N, int C, int H, int W, int K, int stride, int z_x, i
   p.mult = mult; p.s_in = s_in; p.s_Y = s_Y; p.lo_Y = lo_Y; p.hi_Y = hi_Y;
   p.out_dtype = out_dtype;
   const long npix = (long)N * p.Ho * p.Wo;
+  if (C % 4 != 0 || K % 4 != 0) {
+    const long blocks = (npix * K + 127) / 128;
+    if (blocks > 0x7fffffffl) return -2;   // WINO_ERR_UNSUPPORTED: more blocks than a grid holds
+    return launch_kernel(k_direct_conv_bytes, dim3((unsigned)blocks), dim3(128), 0, st, true, p, x, w,
+                         bias, y);
+  }
   if (K % 8 == 0)
     return launch_kernel(k_direct_conv<8>, dim3((unsigned)((npix * (K / 8) + 127) / 128)), dim3(128),
                          0, st, true, p, x, w, bias, y);

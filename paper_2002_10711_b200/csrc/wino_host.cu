@@ -605,7 +605,6 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
   if (d->stride != 1 && d->stride != 2) return WINO_ERR_INVALID;
   if (d->out_dtype != 0 && d->out_dtype != 1) return WINO_ERR_INVALID;
   if (!quant_ok(d->q_x) || !quant_ok(d->q_w) || !quant_ok(d->q_Y)) return WINO_ERR_INVALID;
-  if (d->C % 4 != 0 || d->K % 4 != 0) return WINO_ERR_UNSUPPORTED;
   if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
   const double s_in = (double)d->q_x.scale * (double)d->q_w.scale;

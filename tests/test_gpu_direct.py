@@ -28,7 +28,8 @@ def _run(N, C, H, W, K, stride, q_x, q_w, q_Y, x_q, w_q, bias, out_dtype=0):
 @pytest.mark.parametrize("shape", [(2, 16, 9, 7, 8), (1, 64, 32, 32, 128), (3, 4, 1, 1, 4), (2, 128, 16, 16, 256),
                                    (1, 20, 6, 11, 12),
                                    (3, 128, 8, 8, 64), (5, 64, 4, 4, 96), (1, 256, 5, 19, 32), (2, 192, 1, 1, 64),
-                                   (1, 512, 4, 4, 512), (2, 64, 9, 7, 32)])
+                                   (1, 512, 4, 4, 512), (2, 64, 9, 7, 32),
+                                   (2, 3, 32, 32, 64), (2, 5, 7, 9, 6)])   # any channel count: byte-wise kernel
 @pytest.mark.parametrize("stride", [1, 2])
 @pytest.mark.parametrize("variant", ["plain", "relu_bias", "zero_points"])
 def test_direct_conv_matches_oracle(shape, stride, variant):
@@ -134,5 +135,5 @@ def test_direct_conv_argument_checks():
         binding.direct_conv_forward(1, 16, 8, 8, 16, 3, q, q, q, 16, 16, None, 16, stream=0)
     assert e.value.code == binding.ERR_INVALID
     with pytest.raises(binding.WinoError) as e:
-        binding.direct_conv_forward(1, 6, 8, 8, 16, 1, q, q, q, 16, 16, None, 16, stream=0)
-    assert e.value.code == binding.ERR_UNSUPPORTED
+        binding.direct_conv_forward(1, 8, 8, 8, 16, 1, q, q, q, 16, 24, None, 16, stream=0)   # w not 16-byte aligned
+    assert e.value.code == binding.ERR_ALIGNMENT
