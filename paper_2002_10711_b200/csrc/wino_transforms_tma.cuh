@@ -319,6 +319,18 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     WINO_ST(g_out_trace, trace_step, 1);
     mbar_expect_tx(bar, kInBytes);   // the full box counts, clipped rows included
     tma_load_3d(s_in, &mapM, bar, k0, tau0, 0);
+  } else {
+    griddep_wait();
+  }
+  // while the block's m_q is in flight: this thread's bias in output-code units (a
+  // double-precision division, some forty instructions that would otherwise follow the load)
+  float b_pre[CPT];
+#pragma unroll
+  for (int ch = 0; ch < CPT; ++ch) {
+    const int k = k0 + k4 * CPT + ch;
+    b_pre[ch] = (bias != nullptr && g < ntile) ? (float)((double)__ldg(bias + k) / (double)s_Y) : 0.0f;
+  }
+  if (threadIdx.x == 0) {
     if (!mbar_wait(bar, 0u, &abort_flag)) {
       abort_flag = 1u;
       atomicExch(status, -6);  // WINO_ERR_TIMEOUT
@@ -339,7 +351,6 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     for (int i = 0; i < M * M; ++i) outw[i] = 0u;
 #pragma unroll 1
     for (int ch = 0; ch < CPT; ++ch) {
-      const int k = k0 + k4 * CPT + ch;
       const uint32_t sel_in = 0x7440u | (uint32_t)ch;
       const uint32_t sel_out = insert_selector(ch);
       float Y[M * M];
@@ -349,8 +360,7 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
           mrow[j] = CPT == 1 ? small_int_to_float((int)wd[i * T_ + j])
                              : byte_to_float_sel(wd[i * T_ + j], sel_in, 8388736.0f);
       }, Y);
-      float b_scaled = 0.0f;
-      if (bias != nullptr) b_scaled = (float)((double)__ldg(bias + k) / (double)s_Y);
+      const float b_scaled = b_pre[ch];
 #pragma unroll
       for (int q = 0; q < M * M; ++q) {
         const float yf = __fmaf_rn(Y[q], p.mult_Y, b_scaled);
