@@ -322,8 +322,19 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
   } else {
     griddep_wait();
   }
-  // while the block's m_q is in flight: this thread's bias in output-code units (a
-  // double-precision division, some forty instructions that would otherwise follow the load)
+  // while the block's m_q is in flight: the pixel coordinates of the block's stores (thread 0)
+  // and this thread's bias in output-code units (a double-precision division, some forty
+  // instructions), which would otherwise follow the load
+  int sw[G] = {}, sh[G] = {}, sn[G] = {};
+  if (threadIdx.x == 0) {
+#pragma unroll
+    for (int i = 0; i < G; ++i) {
+      const int tau = tau0 + i;
+      sw[i] = (tau % p.TW) * M;
+      sh[i] = ((tau / p.TW) % p.TH) * M;
+      sn[i] = tau / (p.TW * p.TH);
+    }
+  }
   float b_pre[CPT];
 #pragma unroll
   for (int ch = 0; ch < CPT; ++ch) {
@@ -377,13 +388,9 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
   __syncthreads();
   if (threadIdx.x == 0) {
     WINO_ST(g_out_trace, trace_step, 3);
-    for (int i = 0; i < ntile; ++i) {
-      const int tau = tau0 + i;
-      const int tw = tau % p.TW;
-      const int th = (tau / p.TW) % p.TH;
-      const int n = tau / (p.TW * p.TH);
-      tma_store_4d(&mapY, s_out + (uint32_t)i * kTileOut, k0, tw * M, th * M, n);
-    }
+#pragma unroll
+    for (int i = 0; i < G; ++i)
+      if (i < ntile) tma_store_4d(&mapY, s_out + (uint32_t)i * kTileOut, k0, sw[i], sh[i], sn[i]);
     bulk_commit();
     bulk_wait_all();
     WINO_ST(g_out_trace, trace_step, 4);
