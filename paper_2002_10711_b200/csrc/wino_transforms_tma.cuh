@@ -325,14 +325,14 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
   // while the block's m_q is in flight: the pixel coordinates of the block's stores (thread 0)
   // and this thread's bias in output-code units (a double-precision division, some forty
   // instructions), which would otherwise follow the load
-  int sw[G] = {}, sh[G] = {}, sn[G] = {};
+  __shared__ int store_at[3 * G];   // written and read by thread 0 only (no registers held by the rest)
   if (threadIdx.x == 0) {
 #pragma unroll
     for (int i = 0; i < G; ++i) {
       const int tau = tau0 + i;
-      sw[i] = (tau % p.TW) * M;
-      sh[i] = ((tau / p.TW) % p.TH) * M;
-      sn[i] = tau / (p.TW * p.TH);
+      store_at[3 * i + 0] = (tau % p.TW) * M;
+      store_at[3 * i + 1] = ((tau / p.TW) % p.TH) * M;
+      store_at[3 * i + 2] = tau / (p.TW * p.TH);
     }
   }
   float b_pre[CPT];
@@ -390,7 +390,9 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     WINO_ST(g_out_trace, trace_step, 3);
 #pragma unroll
     for (int i = 0; i < G; ++i)
-      if (i < ntile) tma_store_4d(&mapY, s_out + (uint32_t)i * kTileOut, k0, sw[i], sh[i], sn[i]);
+      if (i < ntile)
+        tma_store_4d(&mapY, s_out + (uint32_t)i * kTileOut, k0, store_at[3 * i], store_at[3 * i + 1],
+                     store_at[3 * i + 2]);
     bulk_commit();
     bulk_wait_all();
     WINO_ST(g_out_trace, trace_step, 4);
