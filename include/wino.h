@@ -75,7 +75,9 @@ enum {
   WINO_ERR_TIMEOUT = -6      /* a bounded device-side wait expired */
 };
 
-/* Execution paths a plan can use (see wino_plan_path / wino_plan_force_path). */
+/* Execution paths a plan can use (see wino_plan_path / wino_plan_force_path).  The automatic
+ * choice is 5 where it applies, else 2 for layers of at most 16 channels in and out, else 1
+ * where C and K are multiples of 16, else 2. */
 enum {
   WINO_PATH_AUTO = 0,
   WINO_PATH_STAGED_TC = 1,   /* transform kernels (TMA-staged where the shape allows) + tcgen05 int8 GEMMs */
