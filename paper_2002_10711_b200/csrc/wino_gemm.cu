@@ -275,15 +275,40 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
       int s = 0, issued = 0; uint32_t ph = 0;
       int xi = blockIdx.x / per_xi, rem = blockIdx.x - xi * per_xi;
       int nb = rem / a.n_mblk, mb = rem - nb * a.n_mblk;
+      // A lone thread retires an instruction every ten to twenty cycles, and the first loads
+      // after the wait are the step's critical path (the generic loop took 0.6 us to get them
+      // out).  So the operands of the first item's first one or two stages are computed, and
+      // pinned in registers, before the wait; after it only the copy instructions themselves
+      // are issued, and the generic loop takes over from there.
+      const int n_first = (KB >= 2 && a.stages >= 2) ? 2 : 1;
+      uint32_t f_bytes = stage_bytes, f_dst = base, f_b_off = (uint32_t)a.MB * a_bytes, f_a_bytes = a_bytes;
+      int f_row_a = (mb * a.MB) * kBM, f_row_b = nb * a.BN, f_xi = xi, f_mb = a.MB, f_n = n_first;
+      asm volatile("" : "+r"(f_bytes), "+r"(f_dst), "+r"(f_b_off), "+r"(f_a_bytes), "+r"(f_row_a),
+                        "+r"(f_row_b), "+r"(f_xi), "+r"(f_mb), "+r"(f_n));
       griddep_wait();
       WINO_ST(g_gemm_trace, trace_step, 2);
+#pragma unroll
+      for (int q = 0; q < 2; ++q) {
+        if (q < f_n) {
+          const uint32_t fb = bar_full + 8u * (uint32_t)q, fd = f_dst + (uint32_t)q * f_bytes;
+          mbar_expect_tx(fb, f_bytes);
+          tma_load_3d(fd, mapV, fb, q * kStageK, f_row_a, f_xi);
+          tma_load_3d(fd + f_b_off, mapU, fb, q * kStageK, f_row_b, f_xi);
+          for (int j = 1; j < f_mb; ++j)   // rows past T are filled with zeros by the TMA unit
+            tma_load_3d(fd + (uint32_t)j * f_a_bytes, mapV, fb, q * kStageK, f_row_a + j * kBM, f_xi);
+          if (q == 0) WINO_ST(g_gemm_trace, trace_step, 15);
+        }
+      }
+      issued = n_first;
+      s = n_first;
+      if (s == a.stages) { s = 0; ph ^= 1u; }
       for (int it = blockIdx.x; it < a.n_items; it += gridDim.x) {
         if (it != blockIdx.x) {
           xi = it / per_xi; rem = it - xi * per_xi;
           nb = rem / a.n_mblk; mb = rem - nb * a.n_mblk;
         }
         bool ok = true;
-        for (int kb = 0; kb < KB; ++kb) {
+        for (int kb = (it == (int)blockIdx.x ? n_first : 0); kb < KB; ++kb) {
           // the ring's first pass finds every stage free
           if (issued >= a.stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
           ++issued;
@@ -294,7 +319,6 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
                         (mb * a.MB + j) * kBM, xi);
           tma_load_3d(sa + (uint32_t)a.MB * a_bytes, mapU, bar_full + 8u * s, kb * kStageK,
                       nb * a.BN, xi);
-          if (it == blockIdx.x && kb == 0) WINO_ST(g_gemm_trace, trace_step, 15);
           if (++s == a.stages) { s = 0; ph ^= 1u; }
         }
         if (!ok) { *abort_p = 1u; break; }
