@@ -94,31 +94,38 @@ k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     if (lane == 0) {
       int s = 0, issued = 0; uint32_t ph = 0;
       griddep_wait();
+      // (a lone thread retires an instruction every ten to twenty cycles, and a stage's MMAs take
+      // about five hundred: everything that does not change inside an item is computed once per
+      // item, and the loops carry running coordinates instead of multiplying)
+      const int n_stages = a.stages, kblocks = a.KB, cb = a.cB, strided = a.stride != 1;
       for (int it = blockIdx.x; it < a.n_items; it += gridDim.x) {
         const int nb = it / n_tiles, tile = it - nb * n_tiles;
         const int tw = tile % a.nW, th = (tile / a.nW) % a.nH, ti = tile / (a.nW * a.nH);
+        const int w0 = tw * a.BW, h0 = th * a.BH, i0 = ti * a.BI, k_row = nb * a.BN;
         bool ok = true;
-        for (int tap = 0; tap < 9 && ok; ++tap) {
-          const int ta = tap / 3, tb = tap - ta * 3;
-          for (int kb = 0; kb < a.KB; ++kb) {
-            if (issued >= a.stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
-            ++issued;
-            const uint32_t sa = base + (uint32_t)s * stage_bytes;
-            mbar_expect_tx(bar_full + 8u * s, stage_bytes);
-            // pixels outside the image (the padding ring, ragged tile edges, images past N)
-            // arrive as zeros
-            if (a.stride == 1) {
-              tma_load_4d(sa, &mapX, bar_full + 8u * s, kb * a.cB, tw * a.BW - 1 + tb, th * a.BH - 1 + ta,
-                          ti * a.BI);
-            } else {
-              // input row 2*ho - 1 + ta: (half-row ho - 1, parity 1), (ho, 0), (ho, 1) for ta = 0, 1, 2
-              const int pcol = tb == 1 ? 0 : 1, dw = tb == 0 ? -1 : 0;
-              const int prow = ta == 1 ? 0 : 1, dh = ta == 0 ? -1 : 0;
-              tma_load_5d(sa, &mapX, bar_full + 8u * s, pcol * a.C + kb * a.cB, tw * a.BW + dw, prow,
-                          th * a.BH + dh, ti * a.BI);
+        int tap = 0;
+        for (int ta = 0; ta < 3 && ok; ++ta) {
+          // stride 1: input row h0 - 1 + ta.  Stride 2: input row 2*ho - 1 + ta, i.e. (half-row
+          // ho - 1, parity 1), (ho, 0), (ho, 1) for ta = 0, 1, 2
+          const int hc = strided ? h0 + (ta == 0 ? -1 : 0) : h0 - 1 + ta;
+          const int prow = ta == 1 ? 0 : 1;
+          for (int tb = 0; tb < 3 && ok; ++tb, ++tap) {
+            const int wc = strided ? w0 + (tb == 0 ? -1 : 0) : w0 - 1 + tb;
+            const int c_base = strided ? (tb == 1 ? 0 : a.C) : 0;
+            int c_off = 0;
+            for (int kb = 0; kb < kblocks; ++kb, c_off += cb) {
+              if (issued >= n_stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
+              ++issued;
+              const uint32_t sa = base + (uint32_t)s * stage_bytes;
+              const uint32_t fb = bar_full + 8u * s;
+              mbar_expect_tx(fb, stage_bytes);
+              // pixels outside the image (the padding ring, ragged tile edges, images past N)
+              // arrive as zeros
+              if (!strided) tma_load_4d(sa, &mapX, fb, c_off, wc, hc, i0);
+              else tma_load_5d(sa, &mapX, fb, c_base + c_off, wc, prow, hc, i0);
+              tma_load_3d(sa + a_bytes, &mapW, fb, c_off, tap, k_row);
+              if (++s == n_stages) { s = 0; ph ^= 1u; }
             }
-            tma_load_3d(sa + a_bytes, &mapW, bar_full + 8u * s, kb * a.cB, tap, nb * a.BN);
-            if (++s == a.stages) { s = 0; ph ^= 1u; }
           }
         }
         if (!ok) { *abort_p = 1u; break; }
