@@ -22,6 +22,7 @@ import os
 import subprocess
 from dataclasses import dataclass, field
 from fractions import Fraction
+from typing import Optional
 
 import numpy as np
 
@@ -51,7 +52,8 @@ class DescC(ct.Structure):
                 ("K", ct.c_int32), ("m", ct.c_int32),
                 ("BT", ct.c_void_p), ("G", ct.c_void_p), ("AT", ct.c_void_p),
                 ("q_x", QuantC), ("q_w", QuantC), ("q_V", QuantC), ("q_U", QuantC),
-                ("q_M", QuantC), ("q_Y", QuantC), ("out_dtype", ct.c_int32)]
+                ("q_M", QuantC), ("q_Y", QuantC), ("out_dtype", ct.c_int32),
+                ("s_w_K", ct.c_void_p), ("s_U_K", ct.c_void_p), ("s_Y_K", ct.c_void_p)]
 
 
 @dataclass
@@ -86,6 +88,10 @@ class Layer:
     q_M: Quant = field(default_factory=Quant)
     q_Y: Quant = field(default_factory=Quant)
     out_dtype: int = 0
+    # per-output-channel scales (K floats) replacing q_w.scale / q_U.scale / q_Y.scale
+    s_w_K: Optional[np.ndarray] = None
+    s_U_K: Optional[np.ndarray] = None
+    s_Y_K: Optional[np.ndarray] = None
 
     @property
     def t(self) -> int:
@@ -134,9 +140,15 @@ class _Keep:
         self.BT, self.G, self.AT = _f32(L.BT), _f32(L.G), _f32(L.AT)
         t = L.t
         assert self.BT.shape == (t, t) and self.G.shape == (t, 3) and self.AT.shape == (L.m, t)
+        self.per_K = []
+        for a in (L.s_w_K, L.s_U_K, L.s_Y_K):
+            if a is not None:
+                a = _f32(a)
+                assert a.shape == (L.K,) and np.all(a > 0)
+            self.per_K.append(a)
         self.d = DescC(L.N, L.C, L.H, L.W, L.K, L.m, _p(self.BT), _p(self.G), _p(self.AT),
                        L.q_x.c(), L.q_w.c(), L.q_V.c(), L.q_U.c(), L.q_M.c(), L.q_Y.c(),
-                       L.out_dtype)
+                       L.out_dtype, _p(self.per_K[0]), _p(self.per_K[1]), _p(self.per_K[2]))
 
     @property
     def ref(self):

@@ -14,6 +14,8 @@
 //   quantize             : rounding table, second implementation via lrintf
 //   staged int8 pipeline : F2 lossless special case == integer direct conv;
 //                          exact-rational recomputation on tiny layers
+//   per-channel scales   : equal scales == per-layer pipeline; every output channel ==
+//                          the per-layer pipeline on that channel alone
 //   flex (perturbed) transforms: parity unpinned beyond the rational
 //                          recomputation within its error bound (no external
 //                          truth exists for a perturbed transform)
@@ -161,7 +163,14 @@ struct Desc {
   const float *BT, *G, *AT;
   Quant q_x, q_w, q_V, q_U, q_M, q_Y;
   int32_t out_dtype;  // 0 = int8, 1 = float
+  // Per-output-channel scales (Section 7 names per-channel quantization as the next
+  // step beyond the per-layer scales of Section 5.1): K floats each, or null for the
+  // per-layer scale of q_w / q_U / q_Y.  Zero points and code ranges stay per layer.
+  const float *s_w_K, *s_U_K, *s_Y_K;
 };
+inline double scale_w(const Desc& d, int k) { return d.s_w_K ? (double)d.s_w_K[k] : (double)d.q_w.scale; }
+inline double scale_U(const Desc& d, int k) { return d.s_U_K ? (double)d.s_U_K[k] : (double)d.q_U.scale; }
+inline double scale_Y(const Desc& d, int k) { return d.s_Y_K ? (double)d.s_Y_K[k] : (double)d.q_Y.scale; }
 
 struct Geo {
   int m, t, TH, TW; long T;
@@ -257,7 +266,8 @@ int32_t orc_quantize(float v, float mult, int32_t z, int32_t qmin, int32_t qmax)
 // double-precision ratio of the stage scales.
 // out[0] = s_x/s_V, out[1] = s_w/s_U, out[2] = s_U*s_V/s_M,
 // out[3] = s_acc/s_Y, out[4] = s_acc, where s_acc = s_M when Q_M is enabled and
-// s_U*s_V otherwise.
+// s_U*s_V otherwise.  Per-layer scales only (per-channel scales, when given, replace
+// s_w, s_U and s_Y by their channel's value in the same formulas).
 void orc_multipliers(const orc_desc_t* d, float* out) {
   double sUV = (double)d->q_U.scale * (double)d->q_V.scale;
   double s_acc = d->q_M.enabled ? (double)d->q_M.scale : sUV;
@@ -305,10 +315,10 @@ int orc_input_stage(const orc_desc_t* d, const int8_t* x_q, float* V_f32, int8_t
 // Stage (2): U = G g G^T for every (k, c) filter, then Q_U (Eq. 1, Fig. 2).
 int orc_weight_stage(const orc_desc_t* d, const int8_t* w_q, float* U_f32, int8_t* U_q) {
   const int t = d->m + 2, C = d->C, K = d->K;
-  const float mult_U = ratio_f32(d->q_w.scale, d->q_U.scale);
 #pragma omp parallel for schedule(static)
   for (int k = 0; k < K; ++k) {
     float gk[9], P[8 * 3], U[64];
+    const float mult_U = ratio_f32(scale_w(*d, k), scale_U(*d, k));
     for (int c = 0; c < C; ++c) {
       for (int a = 0; a < 3; ++a)
         for (int b = 0; b < 3; ++b)
@@ -363,11 +373,13 @@ int orc_hadamard(const orc_desc_t* d, const int8_t* V_q, const int8_t* U_q, int3
 int orc_quantize_M(const orc_desc_t* d, const int32_t* M, int8_t* m_q) {
   Geo g(*d);
   const long total = (long)g.t * g.t * g.T * d->K;
-  const float mult_M =
-      ratio_f32((double)d->q_U.scale * (double)d->q_V.scale, d->q_M.scale);
+  std::vector<float> mult_M((size_t)d->K);   // the accumulator of channel k carries s_U[k] * s_V
+  for (int k = 0; k < d->K; ++k)
+    mult_M[k] = ratio_f32(scale_U(*d, k) * (double)d->q_V.scale, d->q_M.scale);
 #pragma omp parallel for schedule(static)
   for (long i = 0; i < total; ++i)
-    m_q[i] = (int8_t)quantize((float)M[i], mult_M, d->q_M.zero_point, d->q_M.qmin, d->q_M.qmax);
+    m_q[i] = (int8_t)quantize((float)M[i], mult_M[i % d->K], d->q_M.zero_point, d->q_M.qmin,
+                              d->q_M.qmax);
   return 0;
 }
 
@@ -380,9 +392,16 @@ int orc_output_stage(const orc_desc_t* d, const int32_t* M, const int8_t* m_q,
                      const float* bias, float* Y_f32, void* y) {
   Geo g(*d);
   const int t = g.t, m = g.m, K = d->K, H = d->H, W = d->W;
-  float mul[5];
-  orc_multipliers(d, mul);
-  const float mult_Y = mul[3], s_acc = mul[4];
+  // per output channel: s_acc = s_M when Q_M is enabled and s_U[k] * s_V otherwise;
+  // mult_Y = s_acc / s_Y[k]; the bias enters the integer output as bias / s_Y[k]
+  std::vector<float> mult_Y_k((size_t)K), s_acc_k((size_t)K), bias_k((size_t)K);
+  for (int k = 0; k < K; ++k) {
+    const double s_acc_d =
+        d->q_M.enabled ? (double)d->q_M.scale : scale_U(*d, k) * (double)d->q_V.scale;
+    mult_Y_k[k] = ratio_f32(s_acc_d, scale_Y(*d, k));
+    s_acc_k[k] = (float)s_acc_d;
+    bias_k[k] = bias ? (float)((double)bias[k] / scale_Y(*d, k)) : 0.0f;
+  }
 #pragma omp parallel for schedule(static)
   for (long tau = 0; tau < g.T; ++tau) {
     int tw = (int)(tau % g.TW);
@@ -414,10 +433,9 @@ int orc_output_stage(const orc_desc_t* d, const int32_t* M, const int8_t* m_q,
           if (h >= H || w >= W) continue;
           long o = (((long)n * H + h) * W + w) * K + k;
           if (d->out_dtype == 1) {
-            ((float*)y)[o] = std::fmaf(Yv, s_acc, bias ? bias[k] : 0.0f);
+            ((float*)y)[o] = std::fmaf(Yv, s_acc_k[k], bias ? bias[k] : 0.0f);
           } else {
-            float bs = bias ? (float)((double)bias[k] / (double)d->q_Y.scale) : 0.0f;
-            float yf = std::fmaf(Yv, mult_Y, bs);
+            float yf = std::fmaf(Yv, mult_Y_k[k], bias_k[k]);
             ((int8_t*)y)[o] =
                 (int8_t)quantize(yf, 1.0f, d->q_Y.zero_point, d->q_Y.qmin, d->q_Y.qmax);
           }
