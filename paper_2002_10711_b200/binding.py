@@ -25,7 +25,8 @@ STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
 
 EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
-    "wino_plan_force_path", "wino_plan_multipliers", "wino_transform_weights",
+    "wino_plan_force_path", "wino_plan_set_channel_scales", "wino_plan_multipliers",
+    "wino_transform_weights",
     "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward",
     "wino_direct_conv_forward", "wino_direct_last_status", "wino_last_status", "wino_debug_dump_stage",
     "wino_debug_forward_accumulators", "wino_debug_run_stages", "wino_debug_mma_probe",
@@ -74,6 +75,7 @@ def _load() -> ct.CDLL:
     lib.wino_workspace_bytes.restype = sz
     lib.wino_plan_path.argtypes = [vp]
     lib.wino_plan_force_path.argtypes = [vp, i32]
+    lib.wino_plan_set_channel_scales.argtypes = [vp, vp, vp, vp]
     lib.wino_plan_multipliers.argtypes = [vp, vp]
     lib.wino_transform_weights.argtypes = [vp, vp, vp, vp, vp]
     lib.wino_conv_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -175,9 +177,14 @@ class Plan:
 
     @classmethod
     def from_layer(cls, L, **kw):
-        """L: any object with fields N,C,H,W,K,m,BT,G,AT,q_x..q_Y,out_dtype."""
-        return cls(L.N, L.C, L.H, L.W, L.K, L.m, L.BT, L.G, L.AT, L.q_x, L.q_w, L.q_V, L.q_U,
+        """L: any object with fields N,C,H,W,K,m,BT,G,AT,q_x..q_Y,out_dtype and, optionally,
+        per-output-channel scales s_w_K, s_U_K, s_Y_K."""
+        plan = cls(L.N, L.C, L.H, L.W, L.K, L.m, L.BT, L.G, L.AT, L.q_x, L.q_w, L.q_V, L.q_U,
                    L.q_M, L.q_Y, out_dtype=L.out_dtype, **kw)
+        per_K = [getattr(L, n, None) for n in ("s_w_K", "s_U_K", "s_Y_K")]
+        if any(a is not None for a in per_K):
+            plan.set_channel_scales(*per_K)
+        return plan
 
     def __del__(self):
         h = getattr(self, "_h", None)
@@ -200,6 +207,15 @@ class Plan:
 
     def force_path(self, path: int) -> None:
         _check(_lib.wino_plan_force_path(self._h, path), "wino_plan_force_path")
+
+    def set_channel_scales(self, s_w_K=None, s_U_K=None, s_Y_K=None) -> None:
+        """Per-output-channel scales (K floats each; None keeps the per-layer scale)."""
+        keep = [None if a is None else np.ascontiguousarray(a, np.float32) for a in (s_w_K, s_U_K, s_Y_K)]
+        for a in keep:
+            if a is not None and a.shape != (self.K,):
+                raise ValueError("channel scales must have shape (K,)")
+        _check(_lib.wino_plan_set_channel_scales(
+            self._h, *[None if a is None else a.ctypes.data for a in keep]), "wino_plan_set_channel_scales")
 
     def multipliers(self) -> np.ndarray:
         out = np.zeros(5, np.float32)

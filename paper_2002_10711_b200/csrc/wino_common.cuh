@@ -24,6 +24,11 @@ struct Params {
   int qM_enabled;
   int out_dtype;               // 0 int8, 1 float
 };
+// Per-output-channel scales travel beside Params as a device array `chan` [5][K] (null: the
+// per-layer values of Params): row kChMultU = s_w[k]/s_U[k], kChMultM = s_U[k]*s_V/s_M,
+// kChMultY = s_acc[k]/s_Y[k], kChSAcc = s_acc[k] (s_M with Q_M, else s_U[k]*s_V),
+// kChSY = s_Y[k].
+enum { kChMultU = 0, kChMultM = 1, kChMultY = 2, kChSAcc = 3, kChSY = 4 };
 
 // 1.5 * 2^23: adding it to a float of magnitude < 2^22 leaves the
 // round-half-to-even integer in the low mantissa bits.
@@ -41,6 +46,11 @@ __device__ __forceinline__ float quant_magic(float v, float mult, float lo, floa
   return fminf(fmaxf(r, __fadd_rn(lo, kMagic)), __fadd_rn(hi, kMagic));
 }
 __device__ __forceinline__ int magic_to_int(float r) { return __float_as_int(r) - kMagicBits; }
+// Channel k's value of row `row` of the per-channel table, or the per-layer value.
+__device__ __forceinline__ float chan_or(const float* chan, int K, int row, int k,
+                                         float layer_value) {
+  return chan != nullptr ? __ldg(chan + (long)row * K + k) : layer_value;
+}
 
 // Saturating pack of two 32-bit integers to signed bytes (cvt.pack.sat): byte 1 = sat(a),
 // byte 0 = sat(b), upper half = lower half of c.

@@ -22,7 +22,7 @@ namespace wino {
 __global__ void __launch_bounds__(128)
 k_gemm_dp4a(const __grid_constant__ Params p, const int8_t* __restrict__ Vq,
             const int8_t* __restrict__ Uq, void* __restrict__ out, int out_mode,
-            unsigned* __restrict__ absmaxM) {
+            unsigned* __restrict__ absmaxM, const float* __restrict__ chan) {
   const int C4 = p.C >> 2, K4 = p.K >> 2;
   const int xi = blockIdx.z;
   const long idx = blockIdx.x * (long)blockDim.x + threadIdx.x;
@@ -48,7 +48,8 @@ k_gemm_dp4a(const __grid_constant__ Params p, const int8_t* __restrict__ Vq,
       uint32_t wv = 0;
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
-        float r = quant_magic(__int2float_rn(acc[j]), p.mult_M, p.lo_M, p.hi_M);
+        float r = quant_magic(__int2float_rn(acc[j]), chan_or(chan, p.K, kChMultM, k4 * 4 + j, p.mult_M),
+                              p.lo_M, p.hi_M);
         wv |= (__float_as_uint(r) & 0xFFu) << (8 * j);
       }
       *reinterpret_cast<uint32_t*>(reinterpret_cast<int8_t*>(out) + o) = wv;
@@ -64,7 +65,7 @@ int launch_gemm_dp4a(const Params& p, const LaunchOpt& o, const int8_t* Vq, cons
   const long total = (long)p.T * (p.K / 4);
   dim3 grid((unsigned)((total + 127) / 128), 1, (unsigned)(p.t * p.t));
   return launch_kernel(k_gemm_dp4a, grid, dim3(128), 0, st, o.pdl, p, Vq, Uq, out, out_mode,
-                       absmaxM);
+                       absmaxM, o.chan);
 }
 
 // ---------------------------------------------------------------------------
@@ -96,6 +97,7 @@ struct GemmTcArgs {
   int MB;          // m-blocks (128 tiles each) per work item, sharing one U_q tile
   int n_mblk, n_nblk, n_items;   // n_mblk counts groups of MB m-blocks
   int wide_store;  // 1: the output rows are 32-byte aligned (one 256-bit store per row piece)
+  const float* chan;  // per-output-channel multipliers [5][K], or null
 };
 
 template <bool SMALL>
@@ -105,11 +107,12 @@ __device__ __forceinline__ float acc_to_float(uint32_t v) {
 }
 
 // Epilogue of one 32-column chunk of one accumulator row.  FULL: all 32 columns
-// are inside K (no per-element guards).  STATS: track max |M| for calibration.
-template <bool SMALL, bool FULL, bool STATS>
+// are inside K (no per-element guards).  STATS: track max |M| for calibration.  PK: the
+// multiplier of Q_M varies per output channel (column).
+template <bool SMALL, bool FULL, bool STATS, bool PK>
 __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (&r)[32], int k0,
                                                long o, int out_mode, void* out, float& vmax,
-                                               bool wide_store) {
+                                               bool wide_store, const float* chan) {
   if constexpr (STATS) {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -124,7 +127,19 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
   } else {
     uint32_t w[8];
     const float lo_m = __fadd_rn(p.lo_M, kMagic), hi_m = __fadd_rn(p.hi_M, kMagic);
-    if (p.hi_M == 127.0f) {
+    if constexpr (PK) {
+      // every lane reads the same 32 multipliers (one broadcast request per four)
+      const float4* mp = reinterpret_cast<const float4*>(chan + (long)kChMultM * p.K + k0);
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        const float4 mm = (FULL || k0 + q * 4 < p.K) ? __ldg(mp + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const uint32_t b0 = __float_as_uint(quant_magic(acc_to_float<SMALL>(r[4 * q + 0]), mm.x, p.lo_M, p.hi_M));
+        const uint32_t b1 = __float_as_uint(quant_magic(acc_to_float<SMALL>(r[4 * q + 1]), mm.y, p.lo_M, p.hi_M));
+        const uint32_t b2 = __float_as_uint(quant_magic(acc_to_float<SMALL>(r[4 * q + 2]), mm.z, p.lo_M, p.hi_M));
+        const uint32_t b3 = __float_as_uint(quant_magic(acc_to_float<SMALL>(r[4 * q + 3]), mm.w, p.lo_M, p.hi_M));
+        w[q] = __byte_perm(__byte_perm(b0, b1, 0x0040u), __byte_perm(b2, b3, 0x0040u), 0x5410u);
+      }
+    } else if (p.hi_M == 127.0f) {
 #pragma unroll
       for (int q = 0; q < 8; ++q)
         w[q] = quant_pack4<true>(acc_to_float<SMALL>(r[4 * q + 0]), acc_to_float<SMALL>(r[4 * q + 1]),
@@ -151,7 +166,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
 }
 
 // The epilogue warps' loop over their work items.
-template <bool SMALL, bool FULL, bool STATS>
+template <bool SMALL, bool FULL, bool STATS, bool PK = false>
 __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs& a, void* out,
                                               unsigned* absmaxM, uint32_t tmem_base,
                                               uint32_t bar_acc_full, uint32_t bar_acc_empty,
@@ -188,7 +203,7 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
       if (tau >= p.T) continue;
       const int k0 = nb * a.BN + kcol;
       const long o = ((long)xi * p.T + tau) * p.K + k0;
-      epilogue_chunk<SMALL, FULL, STATS>(p, r0, k0, o, a.out_mode, out, vmax, a.wide_store != 0);
+      epilogue_chunk<SMALL, FULL, STATS, PK>(p, r0, k0, o, a.out_mode, out, vmax, a.wide_store != 0, a.chan);
     }
     tc_fence_before();
     __syncwarp();
@@ -377,9 +392,16 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     const bool small = p.C <= 260;
     const bool full = (p.K % a.BN) == 0 && (a.BN % 32) == 0;
     griddep_wait();
-    if (absmaxM != nullptr)
+    const bool per_channel = a.chan != nullptr;
+    if (absmaxM != nullptr && per_channel)
+      epilogue_loop<false, false, true, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
+                                              bar_acc_empty, abort_p, warp, lane, trace_step);
+    else if (absmaxM != nullptr)
       epilogue_loop<false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
                                         abort_p, warp, lane, trace_step);
+    else if (per_channel)
+      epilogue_loop<false, false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
+                                               bar_acc_empty, abort_p, warp, lane, trace_step);
     else if (small && full)
       epilogue_loop<true, true, false>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
                                        abort_p, warp, lane, trace_step);
@@ -439,6 +461,7 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
   a.n_nblk = (p.K + g.BN - 1) / g.BN;
   a.n_items = p.t * p.t * a.n_mblk * a.n_nblk;
   a.wide_store = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
+  a.chan = o.chan;
   return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,
                        mapV, mapU, a, out, absmaxM, status);
 }

@@ -6,6 +6,7 @@
 #include <cstring>
 #include <mutex>
 #include <new>
+#include <vector>
 
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -46,6 +47,7 @@ struct wino_plan {
   bool std_mats;        // BT and AT equal the built-in Cook-Toom matrices bit for bit
   int path;
   int* status_dev;      // device status word (may be null when no GPU is present)
+  float* chan_dev;      // per-output-channel multipliers [5][K] (null: per-layer scales)
   void* kron_dev;       // Kronecker tables of the tensor-core transforms (same allocation)
   unsigned* counters_dev;  // progress counters of the single-launch layer kernel (same allocation)
   CUtensorMap fmapV, fmapU;   // GEMM operand maps of the single-launch kernel
@@ -135,6 +137,10 @@ bool is_std(const float* BT, const float* AT) {
 
 bool path_supported(const wino_plan_t* pl, int path) {
   const int C = pl->d.C, K = pl->d.K;
+  // per-output-channel scales are built into the staged kernels only
+  if (pl->chan_dev != nullptr && path != WINO_PATH_STAGED_TC && path != WINO_PATH_STAGED_TC_PTR &&
+      path != WINO_PATH_STAGED_DP4A)
+    return false;
   switch (path) {
     case WINO_PATH_STAGED_TC:
     case WINO_PATH_STAGED_TC_MMA:
@@ -159,6 +165,7 @@ LaunchOpt opt_of(const wino_plan_t* pl, bool pdl) {
   o.pdl = pdl;
   o.device = pl->device;
   o.num_sms = pl->num_sms;
+  o.chan = pl->chan_dev;
   return o;
 }
 
@@ -393,7 +400,8 @@ int forward_impl(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float
     if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
     rc = launch_output_transform_mma(pl->p, opt_of(pl, pdl), *mm, *my, pl->kron_dev, bias, pl->s_Y,
                                      pl->num_sms, pl->status_dev, st);
-  } else if (tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
+  } else if (tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0 &&
+             pl->chan_dev == nullptr) {   // per-channel output scales: the pointer-based kernel
     const CUtensorMap* mm = map_stage(pl, pl->cache_mld, mbuf, pl->p.K);
     const CUtensorMap* my = map_y(pl, y);
     if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
@@ -540,6 +548,53 @@ int wino_plan_force_path(wino_plan_t* pl, int path) {
   return WINO_OK;
 }
 
+int wino_plan_set_channel_scales(wino_plan_t* pl, const float* s_w_K, const float* s_U_K,
+                                 const float* s_Y_K) {
+  if (pl == nullptr) return WINO_ERR_INVALID;
+  const int K = pl->d.K;
+  if (s_w_K == nullptr && s_U_K == nullptr && s_Y_K == nullptr) {   // back to per-layer scales
+    if (pl->chan_dev) cudaFree(pl->chan_dev);
+    pl->chan_dev = nullptr;
+    return WINO_OK;
+  }
+  for (const float* a : {s_w_K, s_U_K, s_Y_K})
+    if (a != nullptr)
+      for (int k = 0; k < K; ++k)
+        if (!std::isfinite(a[k]) || !(a[k] > 0.0f)) return WINO_ERR_INVALID;
+  if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
+  std::vector<float> tab((size_t)5 * K);
+  const wino_desc_t& d = pl->d;
+  for (int k = 0; k < K; ++k) {
+    const double s_w = s_w_K ? (double)s_w_K[k] : (double)d.q_w.scale;
+    const double s_U = s_U_K ? (double)s_U_K[k] : (double)d.q_U.scale;
+    const double s_Y = s_Y_K ? (double)s_Y_K[k] : (double)d.q_Y.scale;
+    const double sUV = s_U * (double)d.q_V.scale;
+    const double s_acc = d.q_M.enabled ? (double)d.q_M.scale : sUV;
+    tab[(size_t)kChMultU * K + k] = (float)(s_w / s_U);
+    tab[(size_t)kChMultM * K + k] = d.q_M.enabled ? (float)(sUV / (double)d.q_M.scale) : 1.0f;
+    tab[(size_t)kChMultY * K + k] = (float)(s_acc / s_Y);
+    tab[(size_t)kChSAcc * K + k] = (float)s_acc;
+    tab[(size_t)kChSY * K + k] = (float)s_Y;
+  }
+  float* fresh = pl->chan_dev;
+  if (fresh == nullptr && cudaMalloc(&fresh, tab.size() * sizeof(float)) != cudaSuccess) {
+    cudaGetLastError();
+    return WINO_ERR_CUDA;
+  }
+  if (cudaMemcpy(fresh, tab.data(), tab.size() * sizeof(float), cudaMemcpyHostToDevice) !=
+      cudaSuccess) {
+    cudaGetLastError();
+    if (pl->chan_dev == nullptr) cudaFree(fresh);
+    return WINO_ERR_CUDA;
+  }
+  pl->chan_dev = fresh;
+  if (!path_supported(pl, pl->path)) {   // every shape the library plans has a staged path
+    if (path_supported(pl, WINO_PATH_STAGED_TC)) pl->path = WINO_PATH_STAGED_TC;
+    else pl->path = WINO_PATH_STAGED_DP4A;
+  }
+  return WINO_OK;
+}
+
 int wino_plan_multipliers(const wino_plan_t* pl, float out[5]) {
   if (pl == nullptr || out == nullptr) return WINO_ERR_INVALID;
   out[0] = pl->p.mult_V; out[1] = pl->p.mult_U;
@@ -554,7 +609,7 @@ int wino_transform_weights(wino_plan_t* pl, const int8_t* w, int8_t* Uq, uint32_
   if (!aligned16(w) || !aligned16(Uq)) return WINO_ERR_ALIGNMENT;
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
   pl->launches++;
-  return launch_weight_transform(pl->p, w, Uq, absmax, (cudaStream_t)stream);
+  return launch_weight_transform(pl->p, pl->chan_dev, w, Uq, absmax, (cudaStream_t)stream);
 }
 
 int wino_conv_forward(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias,
@@ -748,6 +803,7 @@ long wino_launch_count(const wino_plan_t* pl) { return pl ? pl->launches : 0; }
 void wino_destroy(wino_plan_t* pl) {
   if (pl == nullptr) return;
   if (pl->status_dev) cudaFree(pl->status_dev);
+  if (pl->chan_dev) cudaFree(pl->chan_dev);
   delete pl;
 }
 

@@ -22,6 +22,10 @@ struct LaunchOpt {
   // into L2 while they run.  A hint only; null: none.
   const void* l2_hint = nullptr;
   size_t l2_hint_bytes = 0;   // a multiple of 16
+  // Per-output-channel multipliers, device array [5][K] (rows kChMultU ... kChSY), or null
+  // for the per-layer values of Params.  Read by the weight transform, the GEMM epilogues
+  // and the pointer-based output transform.
+  const float* chan = nullptr;
 };
 
 // "Done once per device" bookkeeping.  cudaFuncSetAttribute applies to the device
@@ -61,8 +65,8 @@ int set_max_smem(DeviceOnce& once, int dev, Kern kernel, size_t smem) {
   });
 }
 
-int launch_weight_transform(const Params& p, const int8_t* w, int8_t* Uq, unsigned* absmax,
-                            cudaStream_t st);
+int launch_weight_transform(const Params& p, const float* chan, const int8_t* w, int8_t* Uq,
+                            unsigned* absmax, cudaStream_t st);
 int launch_input_transform(const Params& p, const LaunchOpt& o, const int8_t* x, int8_t* Vq,
                            unsigned* absmax, cudaStream_t st);
 int launch_output_transform(const Params& p, const LaunchOpt& o, float s_Y, const void* mbuf,

@@ -30,8 +30,9 @@ namespace wino {
 // ---------------------------------------------------------------------------
 template <int M, int CPT>
 __global__ void __launch_bounds__(128)
-k_weight_transform(const __grid_constant__ Params p, const int8_t* __restrict__ w,
-                   int8_t* __restrict__ Uq, unsigned* __restrict__ absmax) {
+k_weight_transform(const __grid_constant__ Params p, const float* __restrict__ chan,
+                   const int8_t* __restrict__ w, int8_t* __restrict__ Uq,
+                   unsigned* __restrict__ absmax) {
   constexpr int T_ = M + 2;
   typedef typename Pack<CPT>::type PT;
   const int CG = p.C / CPT;
@@ -51,6 +52,7 @@ k_weight_transform(const __grid_constant__ Params p, const int8_t* __restrict__ 
 #pragma unroll
     for (int i = 0; i < T_ * T_; ++i) out[i] = 0u;
     const float ubias = 8388736.0f + (float)p.z_w;
+    const float mult_U = chan_or(chan, p.K, kChMultU, k, p.mult_U);
 #pragma unroll
     for (int ch = 0; ch < CPT; ++ch) {
       float g[9];
@@ -74,7 +76,7 @@ k_weight_transform(const __grid_constant__ Params p, const int8_t* __restrict__ 
 #pragma unroll
           for (int l = 0; l < 3; ++l) acc = __fmaf_rn(P[i][l], p.G[j * 3 + l], acc);
           vmax = fmaxf(vmax, fabsf(acc));
-          float r = quant_magic(acc, p.mult_U, p.lo_U, p.hi_U);
+          float r = quant_magic(acc, mult_U, p.lo_U, p.hi_U);
           out[i * T_ + j] = insert_byte(out[i * T_ + j], __float_as_uint(r), ch);
         }
     }
@@ -170,7 +172,7 @@ template <int M, int MODE, bool QM, int CPT, bool STATS>
 __global__ void __launch_bounds__(128)
 k_output_transform(const __grid_constant__ Params p, const void* __restrict__ mbuf,
                    const float* __restrict__ bias, void* __restrict__ y, float s_Y,
-                   unsigned* __restrict__ absmax2) {
+                   unsigned* __restrict__ absmax2, const float* __restrict__ chan) {
   constexpr int T_ = M + 2;
   typedef typename Pack<CPT>::type PT;
   const int KG = p.K / CPT;
@@ -213,8 +215,11 @@ k_output_transform(const __grid_constant__ Params p, const void* __restrict__ mb
         }
       }, Y);
       const float b_real = bias != nullptr ? __ldg(bias + k) : 0.0f;
+      const float mult_Y = chan_or(chan, p.K, kChMultY, k, p.mult_Y);
+      const float s_acc = chan_or(chan, p.K, kChSAcc, k, p.s_acc);
       float b_scaled = 0.0f;
-      if (p.out_dtype == 0 && bias != nullptr) b_scaled = (float)((double)b_real / (double)s_Y);
+      if (p.out_dtype == 0 && bias != nullptr)
+        b_scaled = (float)((double)b_real / (double)chan_or(chan, p.K, kChSY, k, s_Y));
 #pragma unroll
       for (int ip = 0; ip < M; ++ip)
 #pragma unroll
@@ -223,16 +228,16 @@ k_output_transform(const __grid_constant__ Params p, const void* __restrict__ mb
           const int h = th * M + ip, wv = tw * M + jp;
           if constexpr (STATS) {
             ymax = fmaxf(ymax, fabsf(acc));
-            if (h < p.H && wv < p.W) fmax_ = fmaxf(fmax_, fabsf(__fmaf_rn(acc, p.s_acc, b_real)));
+            if (h < p.H && wv < p.W) fmax_ = fmaxf(fmax_, fabsf(__fmaf_rn(acc, s_acc, b_real)));
           }
           if (p.out_dtype == 0) {
-            const float yf = __fmaf_rn(acc, p.mult_Y, b_scaled);
+            const float yf = __fmaf_rn(acc, mult_Y, b_scaled);
             const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
             const uint32_t code = (uint32_t)(magic_to_int(r) + p.z_Y);
             outw[ip * M + jp] = CPT == 1 ? code : __byte_perm(outw[ip * M + jp], code, sel_out);
           } else if (y != nullptr && h < p.H && wv < p.W) {
             reinterpret_cast<float*>(y)[(((long)n * p.H + h) * p.W + wv) * p.K + k] =
-                __fmaf_rn(acc, p.s_acc, b_real);
+                __fmaf_rn(acc, s_acc, b_real);
           }
         }
     }
@@ -267,17 +272,19 @@ int pick_cpt(long items_times_channels) {
 }
 
 template <int M, int CPT>
-int weight_cpt(const Params& p, const int8_t* w, int8_t* Uq, unsigned* absmax, cudaStream_t st) {
+int weight_cpt(const Params& p, const float* chan, const int8_t* w, int8_t* Uq, unsigned* absmax,
+               cudaStream_t st) {
   const long total = (long)p.K * (p.C / CPT);
   return launch_kernel(k_weight_transform<M, CPT>, dim3((unsigned)((total + 127) / 128)), dim3(128),
-                       0, st, false, p, w, Uq, absmax);
+                       0, st, false, p, chan, w, Uq, absmax);
 }
 template <int M>
-int weight_m(const Params& p, const int8_t* w, int8_t* Uq, unsigned* absmax, cudaStream_t st) {
+int weight_m(const Params& p, const float* chan, const int8_t* w, int8_t* Uq, unsigned* absmax,
+             cudaStream_t st) {
   const int cpt = pick_cpt((long)p.K * p.C);
-  return cpt == 4 ? weight_cpt<M, 4>(p, w, Uq, absmax, st)
-       : cpt == 2 ? weight_cpt<M, 2>(p, w, Uq, absmax, st)
-                  : weight_cpt<M, 1>(p, w, Uq, absmax, st);
+  return cpt == 4 ? weight_cpt<M, 4>(p, chan, w, Uq, absmax, st)
+       : cpt == 2 ? weight_cpt<M, 2>(p, chan, w, Uq, absmax, st)
+                  : weight_cpt<M, 1>(p, chan, w, Uq, absmax, st);
 }
 
 template <int M, int MODE, int CPT>
@@ -311,47 +318,47 @@ int input_m(const Params& p, const LaunchOpt& o, const int8_t* x, int8_t* Vq, un
 
 template <int M, int MODE, bool QM, int CPT>
 int output_cpt(const Params& p, bool pdl, float s_Y, const void* mbuf, const float* bias, void* y,
-               unsigned* absmax2, cudaStream_t st) {
+               unsigned* absmax2, const float* chan, cudaStream_t st) {
   const long total = (long)p.T * (p.K / CPT);
   const dim3 grid((unsigned)((total + 127) / 128));
   if constexpr (CPT == 4) {
     if (absmax2 != nullptr)
       return launch_kernel(k_output_transform<M, MODE, QM, 4, true>, grid, dim3(128), 0, st, pdl, p,
-                           mbuf, bias, y, s_Y, absmax2);
+                           mbuf, bias, y, s_Y, absmax2, chan);
   }
   return launch_kernel(k_output_transform<M, MODE, QM, CPT, false>, grid, dim3(128), 0, st, pdl, p,
-                       mbuf, bias, y, s_Y, absmax2);
+                       mbuf, bias, y, s_Y, absmax2, chan);
 }
 template <int M, int MODE, bool QM>
 int output_mode(const Params& p, bool pdl, float s_Y, const void* mbuf, const float* bias, void* y,
-                unsigned* absmax2, cudaStream_t st) {
+                unsigned* absmax2, const float* chan, cudaStream_t st) {
   const int cpt = absmax2 != nullptr ? 4 : pick_cpt((long)p.T * p.K);
-  return cpt == 4 ? output_cpt<M, MODE, QM, 4>(p, pdl, s_Y, mbuf, bias, y, absmax2, st)
-       : cpt == 2 ? output_cpt<M, MODE, QM, 2>(p, pdl, s_Y, mbuf, bias, y, absmax2, st)
-                  : output_cpt<M, MODE, QM, 1>(p, pdl, s_Y, mbuf, bias, y, absmax2, st);
+  return cpt == 4 ? output_cpt<M, MODE, QM, 4>(p, pdl, s_Y, mbuf, bias, y, absmax2, chan, st)
+       : cpt == 2 ? output_cpt<M, MODE, QM, 2>(p, pdl, s_Y, mbuf, bias, y, absmax2, chan, st)
+                  : output_cpt<M, MODE, QM, 1>(p, pdl, s_Y, mbuf, bias, y, absmax2, chan, st);
 }
 template <int M>
 int output_m(const Params& p, const LaunchOpt& o, float s_Y, const void* mbuf, const float* bias,
              void* y, unsigned* absmax2, cudaStream_t st) {
   const bool qm = p.qM_enabled != 0;
   if (!o.std_mats) {
-    return qm ? output_mode<M, kDense, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st)
-              : output_mode<M, kDense, false>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st);
+    return qm ? output_mode<M, kDense, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, o.chan, st)
+              : output_mode<M, kDense, false>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, o.chan, st);
   }
   // With Q_M on, the F4 output transform works on integers in [-128, 127]:
   // every intermediate is an integer below 2^24, so the factored form is exact.
-  if (M != 6 && qm) return output_mode<M, kExact, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st);
-  return qm ? output_mode<M, kSparse, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st)
-            : output_mode<M, kSparse, false>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, st);
+  if (M != 6 && qm) return output_mode<M, kExact, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, o.chan, st);
+  return qm ? output_mode<M, kSparse, true>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, o.chan, st)
+            : output_mode<M, kSparse, false>(p, o.pdl, s_Y, mbuf, bias, y, absmax2, o.chan, st);
 }
 
 }  // namespace
 
 // Entry points for this translation unit's tile size (one unit per m keeps the
 // build parallel).
-int WINO_CAT(launch_weight_transform_m, WINO_M)(const Params& p, const int8_t* w, int8_t* Uq,
-                                                 unsigned* absmax, cudaStream_t st) {
-  return weight_m<WINO_M>(p, w, Uq, absmax, st);
+int WINO_CAT(launch_weight_transform_m, WINO_M)(const Params& p, const float* chan, const int8_t* w,
+                                                 int8_t* Uq, unsigned* absmax, cudaStream_t st) {
+  return weight_m<WINO_M>(p, chan, w, Uq, absmax, st);
 }
 int WINO_CAT(launch_input_transform_m, WINO_M)(const Params& p, const LaunchOpt& o,
                                                 const int8_t* x, int8_t* Vq, unsigned* absmax,

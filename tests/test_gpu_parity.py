@@ -9,7 +9,7 @@ import pytest
 
 import oracle
 import wino_inputs as wi
-from helpers import build_layer, small
+from helpers import build_layer, per_channel, small
 
 pytestmark = pytest.mark.gpu
 
@@ -224,6 +224,81 @@ def test_fused_f2_refuses_other_shapes():
         with pytest.raises(binding.WinoError) as e:
             binding.Plan.from_layer(L, path=FUSED)
         assert e.value.code == binding.ERR_UNSUPPORTED
+
+
+# ---------------------------------------------------------------------------
+# Per-output-channel scales (Section 7) and stage code ranges narrower than eight bits
+# (Section 3.2: every intermediate may have its own bit-width).
+# ---------------------------------------------------------------------------
+PC_SHAPES = [(2, 32, 7, 9, 48), (5, 48, 10, 11, 272), (2, 128, 9, 10, 192), (3, 256, 7, 7, 128)]
+
+
+@pytest.mark.parametrize("m", [2, 4, 6])
+@pytest.mark.parametrize("shape", PC_SHAPES)
+@pytest.mark.parametrize("path", [TC, TC_PTR, DP4A])
+def test_per_channel_scales_every_stage(m, shape, path):
+    N, C, H, W, K = shape
+    wl = wi.Workload("pc", 4000 + m, N, C, H, W, K, m)
+    L, x_q, w_q, bias = build_layer(wl)
+    _compare(per_channel(L, 17 + m, spread=3.0), x_q, w_q, bias, path)
+
+
+@pytest.mark.parametrize("path", [TC, TC_PTR, DP4A])
+@pytest.mark.parametrize("variant", ["no_qm", "float_out", "no_qm_float", "relu", "zero_points", "flex"])
+def test_per_channel_scales_variants(path, variant):
+    wl = wi.Workload("pcv", 4100, 3, 64, 9, 6, 80, 4, flex=(variant == "flex"))
+    L, x_q, w_q, bias = build_layer(wl, q_M=not variant.startswith("no_qm"),
+                                    out_dtype=1 if "float" in variant else 0,
+                                    relu=(variant == "relu"))
+    if variant == "zero_points":
+        L.q_x.zero_point, L.q_w.zero_point, L.q_Y.zero_point = 3, -2, 5
+    _compare(per_channel(L, 23), x_q, w_q, bias, path)
+
+
+def test_per_channel_scales_move_single_kernel_plans_to_a_staged_path():
+    from paper_2002_10711_b200 import binding
+    wl = wi.Workload("pcf", 4200, 2, 64, 8, 8, 64, 2)
+    L, x_q, w_q, bias = build_layer(wl)
+    plan = binding.Plan.from_layer(L)
+    assert plan.path == FUSED
+    P = per_channel(L, 5)
+    plan.set_channel_scales(P.s_w_K, P.s_U_K, P.s_Y_K)
+    assert plan.path == TC
+    for refused in (FUSED, SMALLC, TC_MMA, LAYER):
+        with pytest.raises(binding.WinoError):
+            plan.force_path(refused)
+    plan.set_channel_scales(None, None, None)       # back to per-layer scales
+    plan.force_path(FUSED)
+    with pytest.raises(binding.WinoError):
+        plan.set_channel_scales(np.zeros(L.K, np.float32), None, None)
+    g = _compare(P, x_q, w_q, bias, TC)
+    assert g["launches"] >= 4
+
+
+def test_only_some_channel_scales_given():
+    wl = wi.Workload("pcs", 4300, 2, 32, 6, 6, 32, 4)
+    L, x_q, w_q, bias = build_layer(wl)
+    P = per_channel(L, 9)
+    P.s_U_K = None                                  # weights and output per channel, U per layer
+    _compare(P, x_q, w_q, bias, TC)
+    P = per_channel(L, 10)
+    P.s_w_K = None; P.s_Y_K = None
+    _compare(P, x_q, w_q, bias, DP4A)
+
+
+@pytest.mark.parametrize("path", [TC, TC_PTR, DP4A])
+@pytest.mark.parametrize("m", [2, 4, 6])
+def test_narrow_code_ranges_per_stage(path, m):
+    """6-bit V, 5-bit U, 7-bit M and a 4-bit output, each with its own calibrated-then-widened
+    scale: clamps at every stage, identical codes."""
+    wl = wi.Workload("bits", 4400 + m, 3, 48, 9, 7, 64, m)
+    L, x_q, w_q, bias = build_layer(wl)
+    for q, bits in ((L.q_V, 6), (L.q_U, 5), (L.q_M, 7), (L.q_Y, 4)):
+        top = 2 ** (bits - 1) - 1
+        q.scale = float(np.float32(q.scale * 127.0 / top * 0.8))   # 0.8: some values clip
+        q.qmin, q.qmax = -top, top
+    g = _compare(L, x_q, w_q, bias, path)
+    assert np.abs(g["V_q"]).max() == 31 and np.abs(g["y"]).max() == 7
 
 
 def test_saturating_scales_clip_identically():
