@@ -201,7 +201,7 @@ def aggregate(ms_local: float, units_local: float, dist=None):
 
 
 def time_layer_quick(binding, cook_toom, torch, dev, N, C, H, W, K, m, flex_seed=None, path=0,
-                     steps=96):
+                     steps=96, channel_scales=False):
     """Steady-state microseconds per forward call of one layer shape on rotating buffers
     (more bytes than L2), from a CUDA graph, with fixed stage scales: the kernels have no
     data-dependent control flow, so for timing the values and scales do not matter.
@@ -215,6 +215,9 @@ def time_layer_quick(binding, cook_toom, torch, dev, N, C, H, W, K, m, flex_seed
     try:
         plan = binding.Plan(N, C, H, W, K, m, BT, G, AT, q(1 / 32), q(0.004), q(0.5), q(0.01),
                             q(30.0), q(100.0), path=path)
+        if channel_scales:   # per-output-channel scales for w, U and y (seeded factors)
+            f_w, f_U, f_Y = wi.channel_factors(7, K)
+            plan.set_channel_scales(0.004 * f_w, 0.01 * f_U, 100.0 * f_Y)
     except binding.WinoError as e:
         return None, str(e)
     xb, yb = N * H * W * C, N * H * W * K
@@ -679,6 +682,13 @@ def run_ours(args, wl):
                                        flex_seed=o.seed if o.flex else None)
             if us is not None:
                 other.append(layer_row(peaks, name, o.N, o.C, o.H, o.W, o.K, o.m, us, pth))
+        # the headline layer with per-output-channel scales (staged path, pointer-based
+        # output transform)
+        us, pth = time_layer_quick(binding, cook_toom, torch, dev, wl.N, wl.C, wl.H, wl.W, wl.K, wl.m,
+                                   channel_scales=True)
+        if us is not None:
+            other.append(layer_row(peaks, wl.name + ".per_channel_scales", wl.N, wl.C, wl.H, wl.W,
+                                   wl.K, wl.m, us, pth))
         for ly in wi.resnet18_layers(1005, 256):
             if ly["m"] == 0:
                 continue      # stride-2 layers are direct convolutions, not timed

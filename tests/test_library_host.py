@@ -123,3 +123,23 @@ def test_once_per_device_bookkeeping():
     assert binding.debug_once_per_device(63) == 1
     assert binding.debug_once_per_device(64) == binding.ERR_INVALID
     assert binding.debug_once_per_device(-1) == binding.ERR_INVALID
+
+
+def test_channel_scales_are_validated_on_the_host():
+    p = _plan(C=64, K=64, m=2)            # a layer the fused F2 kernel would take
+    ok = np.full(64, 0.1, np.float32)
+    bad = ok.copy(); bad[7] = 0.0
+    nan = ok.copy(); nan[3] = np.nan
+    lib = binding._lib
+    for arr in (bad, nan, -ok):
+        assert lib.wino_plan_set_channel_scales(p._h, arr.ctypes.data, None, None) == binding.ERR_INVALID
+        assert lib.wino_plan_set_channel_scales(p._h, None, None, arr.ctypes.data) == binding.ERR_INVALID
+    before = p.path
+    assert lib.wino_plan_set_channel_scales(p._h, None, None, None) == binding.WINO_OK   # nothing to undo
+    assert p.path == before
+    with pytest.raises(ValueError):
+        p.set_channel_scales(np.ones(3, np.float32))
+    rc = lib.wino_plan_set_channel_scales(p._h, ok.ctypes.data, None, None)
+    assert rc in (binding.WINO_OK, binding.ERR_CUDA)      # needs a device for its table
+    if rc == binding.WINO_OK:
+        assert p.path == binding.PATH_STAGED_TC
