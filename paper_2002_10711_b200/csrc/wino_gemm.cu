@@ -98,6 +98,7 @@ struct GemmTcArgs {
   int n_mblk, n_nblk, n_items;   // n_mblk counts groups of MB m-blocks
   int wide_store;  // 1: the output rows are 32-byte aligned (one 256-bit store per row piece)
   const float* chan;  // per-output-channel multipliers [5][K], or null
+  int chan_smem;      // 1: the block keeps the K multipliers of Q_M in shared memory
 };
 
 template <bool SMALL>
@@ -112,7 +113,7 @@ __device__ __forceinline__ float acc_to_float(uint32_t v) {
 template <bool SMALL, bool FULL, bool STATS, bool PK>
 __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (&r)[32], int k0,
                                                long o, int out_mode, void* out, float& vmax,
-                                               bool wide_store, const float* chan) {
+                                               bool wide_store, const float* mult_k) {
   if constexpr (STATS) {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -128,11 +129,20 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
     uint32_t w[8];
     const float lo_m = __fadd_rn(p.lo_M, kMagic), hi_m = __fadd_rn(p.hi_M, kMagic);
     if constexpr (PK) {
-      // every lane reads the same 32 multipliers (one broadcast request per four)
-      const float4* mp = reinterpret_cast<const float4*>(chan + (long)kChMultM * p.K + k0);
+      // every lane reads the same 32 multipliers (one broadcast request per four); mult_k
+      // is the block's copy in shared memory, or the table in global memory
+      const float4* mp = reinterpret_cast<const float4*>(mult_k + k0);
 #pragma unroll
       for (int q = 0; q < 8; ++q) {
-        const float4 mm = (FULL || k0 + q * 4 < p.K) ? __ldg(mp + q) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 mm = (FULL || k0 + q * 4 < p.K) ? mp[q] : make_float4(0.f, 0.f, 0.f, 0.f);
+        if (p.hi_M == 127.0f) {   // upper bound by the saturating pack, as in quant_pack4
+          const int c0 = magic_to_int(fmaxf(__fmaf_rn(acc_to_float<SMALL>(r[4 * q + 0]), mm.x, kMagic), lo_m));
+          const int c1 = magic_to_int(fmaxf(__fmaf_rn(acc_to_float<SMALL>(r[4 * q + 1]), mm.y, kMagic), lo_m));
+          const int c2 = magic_to_int(fmaxf(__fmaf_rn(acc_to_float<SMALL>(r[4 * q + 2]), mm.z, kMagic), lo_m));
+          const int c3 = magic_to_int(fmaxf(__fmaf_rn(acc_to_float<SMALL>(r[4 * q + 3]), mm.w, kMagic), lo_m));
+          w[q] = pack_sat_s8(c1, c0, pack_sat_s8(c3, c2, 0u));
+          continue;
+        }
         const uint32_t b0 = __float_as_uint(quant_magic(acc_to_float<SMALL>(r[4 * q + 0]), mm.x, p.lo_M, p.hi_M));
         const uint32_t b1 = __float_as_uint(quant_magic(acc_to_float<SMALL>(r[4 * q + 1]), mm.y, p.lo_M, p.hi_M));
         const uint32_t b2 = __float_as_uint(quant_magic(acc_to_float<SMALL>(r[4 * q + 2]), mm.z, p.lo_M, p.hi_M));
@@ -171,7 +181,7 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
                                               unsigned* absmaxM, uint32_t tmem_base,
                                               uint32_t bar_acc_full, uint32_t bar_acc_empty,
                                               volatile uint32_t* abort_p, int warp, int lane,
-                                              int trace_step) {
+                                              int trace_step, const float* mult_k = nullptr) {
   (void)trace_step;
   const int quad = warp & 3;
   const int sub = (warp - 2) >> 2;
@@ -203,7 +213,7 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
       if (tau >= p.T) continue;
       const int k0 = nb * a.BN + kcol;
       const long o = ((long)xi * p.T + tau) * p.K + k0;
-      epilogue_chunk<SMALL, FULL, STATS, PK>(p, r0, k0, o, a.out_mode, out, vmax, a.wide_store != 0, a.chan);
+      epilogue_chunk<SMALL, FULL, STATS, PK>(p, r0, k0, o, a.out_mode, out, vmax, a.wide_store != 0, mult_k);
     }
     tc_fence_before();
     __syncwarp();
@@ -213,12 +223,13 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
   if constexpr (STATS) atomic_absmax(absmaxM, vmax);
 }
 
-__global__ void __launch_bounds__(kGemmThreads, 1)
-k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV_param,
-          const __grid_constant__ CUtensorMap mapU_param, const GemmTcArgs a, void* __restrict__ out,
-          unsigned* __restrict__ absmaxM, int* __restrict__ status) {
-  const CUtensorMap* mapV = &mapV_param;
-  const CUtensorMap* mapU = &mapU_param;
+// PK: Q_M takes one multiplier per output channel (a build of its own, so that the
+// per-layer kernel carries none of that code).
+template <bool PK>
+__device__ __forceinline__ void gemm_tc_body(const Params& p, const CUtensorMap* mapV,
+                                             const CUtensorMap* mapU, const GemmTcArgs& a,
+                                             void* __restrict__ out, unsigned* __restrict__ absmaxM,
+                                             int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -391,17 +402,33 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     // of every column block lies inside K (the last block is not ragged).
     const bool small = p.C <= 260;
     const bool full = (p.K % a.BN) == 0 && (a.BN % 32) == 0;
+    const bool per_channel = PK;
+    // Per-channel multipliers of Q_M: the block's own copy in shared memory (the L1 left
+    // beside 200 KB of operand ring does not keep the table while the epilogue's stores
+    // stream through it).  The table is written by the host before any launch, so it is
+    // read ahead of the dependency wait.
+    const float* mult_k = PK ? a.chan + (long)kChMultM * p.K : nullptr;
+    if (PK && a.chan_smem) {
+      float* tab = reinterpret_cast<float*>(gen + (bars + 16u * (uint32_t)a.stages + 64u - base));
+      for (int i = (int)threadIdx.x - 64; i < p.K; i += 32 * kEpiWarps) tab[i] = __ldg(mult_k + i);
+      asm volatile("bar.sync 1, %0;" ::"n"(32 * kEpiWarps) : "memory");
+      mult_k = tab;
+    }
     griddep_wait();
-    const bool per_channel = a.chan != nullptr;
-    if (absmaxM != nullptr && per_channel)
-      epilogue_loop<false, false, true, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
-                                              bar_acc_empty, abort_p, warp, lane, trace_step);
-    else if (absmaxM != nullptr)
+    if constexpr (PK) {
+      (void)per_channel;
+      if (absmaxM != nullptr)
+        epilogue_loop<false, false, true, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
+                                                bar_acc_empty, abort_p, warp, lane, trace_step, mult_k);
+      else if (small && full)
+        epilogue_loop<true, true, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
+                                               bar_acc_empty, abort_p, warp, lane, trace_step, mult_k);
+      else
+        epilogue_loop<false, false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
+                                                 bar_acc_empty, abort_p, warp, lane, trace_step, mult_k);
+    } else if (absmaxM != nullptr)
       epilogue_loop<false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
                                         abort_p, warp, lane, trace_step);
-    else if (per_channel)
-      epilogue_loop<false, false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
-                                               bar_acc_empty, abort_p, warp, lane, trace_step);
     else if (small && full)
       epilogue_loop<true, true, false>(p, a, out, absmaxM, tmem_base, bar_acc_full, bar_acc_empty,
                                        abort_p, warp, lane, trace_step);
@@ -421,6 +448,20 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
   }
+}
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV,
+          const __grid_constant__ CUtensorMap mapU, const GemmTcArgs a, void* __restrict__ out,
+          unsigned* __restrict__ absmaxM, int* __restrict__ status) {
+  gemm_tc_body<false>(p, &mapV, &mapU, a, out, absmaxM, status);
+}
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_tc_per_channel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV,
+                      const __grid_constant__ CUtensorMap mapU, const GemmTcArgs a,
+                      void* __restrict__ out, unsigned* __restrict__ absmaxM,
+                      int* __restrict__ status) {
+  gemm_tc_body<true>(p, &mapV, &mapU, a, out, absmaxM, status);
 }
 
 TcGeom tc_geometry(const Params& p, int num_sms) {
@@ -462,6 +503,15 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
   a.n_items = p.t * p.t * a.n_mblk * a.n_nblk;
   a.wide_store = (reinterpret_cast<uintptr_t>(out) & 31u) == 0 ? 1 : 0;
   a.chan = o.chan;
+  // room for the multipliers behind the ring and the barriers (the ring stops at 196 KB)
+  a.chan_smem = (o.chan != nullptr && (size_t)p.K * 4 <= 24 * 1024) ? 1 : 0;
+  if (o.chan != nullptr) {
+    static DeviceOnce once_pk;
+    if (int rc = set_max_smem(once_pk, o.device, k_gemm_tc_per_channel, 227 * 1024)) return rc;
+    const size_t smem = g.smem + (a.chan_smem ? (size_t)p.K * 4 : 0);
+    return launch_kernel(k_gemm_tc_per_channel, dim3((unsigned)g.grid), dim3(kGemmThreads), smem, st,
+                         o.pdl, p, mapV, mapU, a, out, absmaxM, status);
+  }
   return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,
                        mapV, mapU, a, out, absmaxM, status);
 }

@@ -400,8 +400,7 @@ int forward_impl(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float
     if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;
     rc = launch_output_transform_mma(pl->p, opt_of(pl, pdl), *mm, *my, pl->kron_dev, bias, pl->s_Y,
                                      pl->num_sms, pl->status_dev, st);
-  } else if (tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0 &&
-             pl->chan_dev == nullptr) {   // per-channel output scales: the pointer-based kernel
+  } else if (tma_ok && pl->p.qM_enabled && pl->p.out_dtype == 0 && tma_chunk(pl->p.K) != 0) {
     const CUtensorMap* mm = map_stage(pl, pl->cache_mld, mbuf, pl->p.K);
     const CUtensorMap* my = map_y(pl, y);
     if (mm == nullptr || my == nullptr) return WINO_ERR_CUDA;

@@ -24,7 +24,7 @@ struct LaunchOpt {
   size_t l2_hint_bytes = 0;   // a multiple of 16
   // Per-output-channel multipliers, device array [5][K] (rows kChMultU ... kChSY), or null
   // for the per-layer values of Params.  Read by the weight transform, the GEMM epilogues
-  // and the pointer-based output transform.
+  // and the output transforms.
   const float* chan = nullptr;
 };
 

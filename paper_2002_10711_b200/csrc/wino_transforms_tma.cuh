@@ -276,11 +276,14 @@ k_input_transform_tma_multi(const __grid_constant__ Params p, const __grid_const
   if (threadIdx.x == 0) bulk_wait_all();
 }
 
-template <int M, int MODE, int KC, int G, int CPT>
+// PK: the output scale varies per output channel (`chan`, rows kChMultY and kChSY; one
+// channel per thread only).
+template <int M, int MODE, int KC, int G, int CPT, bool PK = false>
 __global__ void __launch_bounds__((KC / CPT) * G, tma_min_blocks((KC / CPT) * G, CPT, M <= 4))
 k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapM,
                        const __grid_constant__ CUtensorMap mapY, const float* __restrict__ bias,
-                       float s_Y, int* __restrict__ status) {
+                       float s_Y, int* __restrict__ status, const float* __restrict__ chan) {
+  static_assert(!PK || CPT == 1, "per-channel scales: one channel per thread");
   constexpr int T_ = M + 2, T2 = T_ * T_, TPT = KC / CPT;
   constexpr uint32_t kInBytes = T2 * G * KC;          // [T2][G][KC]
   constexpr uint32_t kTileOutBytes = M * M * KC;      // [M][M][KC] per tile
@@ -336,6 +339,11 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
     }
   }
   float b_pre[CPT];
+  float mult_Y = p.mult_Y;
+  if constexpr (PK) {
+    mult_Y = __ldg(chan + (long)kChMultY * p.K + k0 + k4);
+    s_Y = __ldg(chan + (long)kChSY * p.K + k0 + k4);
+  }
 #pragma unroll
   for (int ch = 0; ch < CPT; ++ch) {
     const int k = k0 + k4 * CPT + ch;
@@ -374,7 +382,7 @@ k_output_transform_tma(const __grid_constant__ Params p, const __grid_constant__
       const float b_scaled = b_pre[ch];
 #pragma unroll
       for (int q = 0; q < M * M; ++q) {
-        const float yf = __fmaf_rn(Y[q], p.mult_Y, b_scaled);
+        const float yf = __fmaf_rn(Y[q], PK ? mult_Y : p.mult_Y, b_scaled);
         const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
         const uint32_t code = (uint32_t)(magic_to_int(r) + p.z_Y);
         outw[q] = CPT == 1 ? code : __byte_perm(outw[q], code, sel_out);
@@ -491,20 +499,26 @@ int input_tma_mode(const Params& p, const LaunchOpt& o, const CUtensorMap& mapX,
                     : input_tma_launch<M, MODE, 16, 8, 2>(p, o, mapX, mapV, status, st);
 }
 
-template <int M, int MODE, int KC, int G, int CPT>
+template <int M, int MODE, int KC, int G, int CPT, bool PK = false>
 int output_tma_launch(const Params& p, const LaunchOpt& o, const CUtensorMap& mapM, const CUtensorMap& mapY,
                       const float* bias, float s_Y, int* status, cudaStream_t st) {
   constexpr size_t smem = (size_t)G * ((M + 2) * (M + 2) * KC + ((M * M * KC + 127) / 128 * 128)) + 128 + 16;
   static DeviceOnce once;   // one per instantiation
-  if (int rc = set_max_smem(once, o.device, k_output_transform_tma<M, MODE, KC, G, CPT>, smem)) return rc;
+  if (int rc = set_max_smem(once, o.device, k_output_transform_tma<M, MODE, KC, G, CPT, PK>, smem)) return rc;
   const int units = ((p.T + G - 1) / G) * (p.K / KC);
-  return launch_kernel(k_output_transform_tma<M, MODE, KC, G, CPT>, dim3((unsigned)units),
-                       dim3((KC / CPT) * G), smem, st, o.pdl, p, mapM, mapY, bias, s_Y, status);
+  return launch_kernel(k_output_transform_tma<M, MODE, KC, G, CPT, PK>, dim3((unsigned)units),
+                       dim3((KC / CPT) * G), smem, st, o.pdl, p, mapM, mapY, bias, s_Y, status,
+                       PK ? o.chan : nullptr);
 }
 template <int M, int MODE>
 int output_tma_mode(const Params& p, const LaunchOpt& o, const CUtensorMap& mapM, const CUtensorMap& mapY,
                     const float* bias, float s_Y, int* status, cudaStream_t st) {
   const int kc = tma_chunk(p.K);
+  if (o.chan != nullptr)   // per-output-channel scales: the one-channel-per-thread build
+    return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 1, true>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 1, true>(p, o, mapM, mapY, bias, s_Y, status, st)
+         : kc == 32 ? output_tma_launch<M, MODE, 32, 4, 1, true>(p, o, mapM, mapY, bias, s_Y, status, st)
+                    : output_tma_launch<M, MODE, 16, 8, 1, true>(p, o, mapM, mapY, bias, s_Y, status, st);
   if (tma_cpt((long)p.T * p.K) == 4)
     return kc == 128 ? output_tma_launch<M, MODE, 128, 1, 4>(p, o, mapM, mapY, bias, s_Y, status, st)
          : kc == 64 ? output_tma_launch<M, MODE, 64, 4, 4>(p, o, mapM, mapY, bias, s_Y, status, st)
