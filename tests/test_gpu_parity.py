@@ -356,6 +356,38 @@ def test_gpu_calibration_matches_oracle_calibration():
         assert tuple(np.float32(got)) == tuple(np.float32(want)), (name, got, want)
 
 
+@pytest.mark.parametrize("path", [TC, DP4A])
+def test_calibration_statistics_with_channel_scales(path):
+    """The four max-abs statistics of a calibration pass on a plan with per-channel scales,
+    against the same maxima taken over the oracle's stage outputs."""
+    import copy
+    import torch
+    from paper_2002_10711_b200 import binding
+    wl = wi.Workload("pccal", 4500, 3, 64, 9, 7, 80, 4)
+    L, x_q, w_q, bias = build_layer(wl)
+    P = per_channel(L, 41, spread=3.0)
+    plan = binding.Plan.from_layer(P, path=path)
+    x = torch.from_numpy(x_q).cuda()
+    w = torch.from_numpy(w_q).cuda()
+    b = torch.from_numpy(bias).cuda()
+    U = torch.empty(plan.weight_bytes, dtype=torch.int8, device="cuda")
+    ws = torch.empty(plan.workspace_bytes, dtype=torch.uint8, device="cuda")
+    stats = torch.zeros(4, dtype=torch.int32, device="cuda")
+    plan.transform_weights(w, U)
+    plan.calibrate_forward(x, U, b, None, ws, stats)
+    assert plan.last_status() == 0
+    got = stats.cpu().numpy().view(np.float32)
+    _, Vf = oracle.input_stage(P, x_q, want_f32=True)
+    _, d = oracle.forward(P, x_q, w_q, bias=bias, dumps=True)
+    _, Yf = oracle.output_stage(P, d["M"], d["m_q"], bias, want_f32=True)
+    F = copy.deepcopy(P)
+    F.out_dtype = 1
+    y_float = oracle.forward(F, x_q, w_q, bias=bias)
+    want = np.array([np.abs(Vf).max(), np.abs(d["M"]).max(), np.abs(Yf).max(), np.abs(y_float).max()],
+                    np.float32)
+    assert (got.view(np.uint32) == want.view(np.uint32)).all(), (got, want)
+
+
 def test_mma_probe_runs_and_reports_ok():
     import torch
     from paper_2002_10711_b200 import binding, cook_toom
