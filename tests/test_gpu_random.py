@@ -6,7 +6,7 @@ import pytest
 
 import oracle
 import wino_inputs as wi
-from helpers import build_layer
+from helpers import build_layer, per_channel
 
 pytestmark = pytest.mark.gpu
 
@@ -26,12 +26,12 @@ def _cases(n, seed):
                         q_M=bool(d[7] % np.uint64(4)), out_dtype=int(d[8] % np.uint64(4) == 0),
                         relu=bool(d[9] & np.uint64(1)), with_bias=bool(d[10] % np.uint64(3)),
                         zp=bool(d[11] % np.uint64(4) == 0), path_draw=int(d[12] % np.uint64(97)),
-                        seed=int(d[13] % np.uint64(100000))))
+                        seed=int(d[13] % np.uint64(100000)),
+                        per_channel=bool(d[14] % np.uint64(3) == 0)))
     return out
 
 
-@pytest.mark.parametrize("case", _cases(48, 20260), ids=lambda c: f"m{c['m']}C{c['C']}K{c['K']}H{c['H']}W{c['W']}")
-def test_random_layer(case):
+def check_case(case):
     from gpu_helpers import gpu_run
     from paper_2002_10711_b200 import binding
     wl = wi.Workload("r", case["seed"], case["N"], case["C"], case["H"], case["W"], case["K"], case["m"],
@@ -40,8 +40,11 @@ def test_random_layer(case):
                                     with_bias=case["with_bias"])
     if case["zp"]:
         L.q_x.zero_point, L.q_w.zero_point, L.q_Y.zero_point = 3, -2, 5
+    if case["per_channel"]:
+        L = per_channel(L, case["seed"] + 1, spread=3.0)
     supported = []
-    for path in (1, 2, 3, 4, 5):
+    # per-channel scales exist on the staged paths; a plan forced elsewhere moves to one
+    for path in ((1, 2, 4) if case["per_channel"] else (1, 2, 3, 4, 5, 6, 7)):
         try:
             binding.Plan.from_layer(L, path=path)
             supported.append(path)
@@ -61,3 +64,8 @@ def test_random_layer(case):
     g2 = gpu_run(L, x_q, w_q, bias)
     if L.out_dtype == 0:
         assert (g2["y"] == y_ref).all(), (case, "auto", g2["path"])
+
+
+@pytest.mark.parametrize("case", _cases(64, 20260), ids=lambda c: f"m{c['m']}C{c['C']}K{c['K']}H{c['H']}W{c['W']}")
+def test_random_layer(case):
+    check_case(case)
