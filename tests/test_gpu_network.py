@@ -20,7 +20,7 @@ def _weights(seed, idx, K, C):
     return wi.gaussian_weight_codes(seed, 100 + idx, (K, 3, 3, C), float(np.sqrt(2.0 / (9 * C))))
 
 
-def _run_chain(batch):
+def _run_chain(batch, per_channel_weights=False):
     from gpu_helpers import gpu_run
     seed = 1005
     layers = wi.resnet18_layers(seed, batch)
@@ -56,6 +56,12 @@ def _run_chain(batch):
         L.q_w = Quant(scale=float(s_w))
         L.q_Y = Quant(qmin=0)
         L = calibrate(L, x_ref, w_q, None)
+        if per_channel_weights:
+            # weights and transformed weights scaled per output channel, activations per
+            # layer (the next layer sums over these channels, so its input has one scale)
+            f_w, f_U, _ = wi.channel_factors(seed + spec["index"], spec["K"], 1.5)
+            L.s_w_K = (np.float32(L.q_w.scale) * f_w).astype(np.float32)
+            L.s_U_K = (np.float32(L.q_U.scale) * f_U).astype(np.float32)
         y_ref = oracle.forward(L, x_ref, w_q)
         g1 = gpu_run(L, x_ref, w_q, None)
         assert (g1["y"] == y_ref).all(), f"layer {spec['index']} (oracle-fed) differs"
@@ -68,6 +74,11 @@ def _run_chain(batch):
 
 def test_resnet18_chain_small_batch():
     seen = _run_chain(4)
+    assert seen == {2, 4, 6}
+
+
+def test_resnet18_chain_with_per_channel_weight_scales():
+    seen = _run_chain(4, per_channel_weights=True)
     assert seen == {2, 4, 6}
 
 
