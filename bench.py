@@ -215,9 +215,9 @@ def time_layer_quick(binding, cook_toom, torch, dev, N, C, H, W, K, m, flex_seed
     try:
         plan = binding.Plan(N, C, H, W, K, m, BT, G, AT, q(1 / 32), q(0.004), q(0.5), q(0.01),
                             q(30.0), q(100.0), path=path)
-        if channel_scales:   # per-output-channel scales for w, U and y (seeded factors)
-            f_w, f_U, f_Y = wi.channel_factors(7, K)
-            plan.set_channel_scales(0.004 * f_w, 0.01 * f_U, 100.0 * f_Y)
+        if channel_scales:   # per-output-channel scales for w, U, M and y (seeded factors)
+            f_w, f_U, f_M, f_Y = wi.channel_factors(7, K)
+            plan.set_channel_scales(0.004 * f_w, 0.01 * f_U, 30.0 * f_M, 100.0 * f_Y)
     except binding.WinoError as e:
         return None, str(e)
     xb, yb = N * H * W * C, N * H * W * K

@@ -147,20 +147,22 @@ int wino_plan_force_path(wino_plan_t* plan, int path);
 
 /* Per-output-channel scales (paper: Section 7 names per-channel quantization as the step
  * beyond the per-layer scales of Section 5.1).  Each argument is a HOST array of K positive
- * finite floats, copied by the call, or NULL to keep the descriptor's per-layer scale:
- * s_w_K[k] replaces q_w.scale for filter k, s_U_K[k] replaces q_U.scale for the transformed
- * filter k (so the Hadamard sums of channel k carry s_U_K[k] * q_V.scale and Q_M uses one
- * multiplier per channel), s_Y_K[k] replaces q_Y.scale for output channel k (the bias enters
- * the integer output as bias[k] / s_Y_K[k]).  Zero points and code ranges stay per layer.
- * All three NULL returns the plan to per-layer scales.  Call before wino_transform_weights;
- * U_q made under other scales is stale.  The staged paths (WINO_PATH_STAGED_TC,
- * WINO_PATH_STAGED_TC_PTR, WINO_PATH_STAGED_DP4A) implement it: a plan on another path moves
- * to the staged tcgen05 path (or the staged dp4a path), forcing another path afterwards
- * returns WINO_ERR_UNSUPPORTED, and wino_plan_multipliers keeps reporting the per-layer
- * values.  Synchronous (one small host-to-device copy); WINO_ERR_INVALID for a bad scale,
- * WINO_ERR_CUDA without a device. */
+ * finite floats, copied by the call, or NULL to keep the descriptor's per-layer scale, for
+ * the four tensors that carry the output-channel axis: s_w_K[k] replaces q_w.scale for
+ * filter k, s_U_K[k] replaces q_U.scale for the transformed filter k (so the Hadamard sums
+ * of channel k carry s_U_K[k] * q_V.scale), s_M_K[k] replaces q_M.scale for channel k of the
+ * quantized Hadamard sums (ignored when q_M is disabled), s_Y_K[k] replaces q_Y.scale for
+ * output channel k (the bias enters the integer output as bias[k] / s_Y_K[k]).  The input
+ * side (x, V) is summed over its channels and keeps one scale; zero points and code ranges
+ * stay per layer.  All four NULL returns the plan to per-layer scales.  Call before
+ * wino_transform_weights; U_q made under other scales is stale.  The staged paths
+ * (WINO_PATH_STAGED_TC, WINO_PATH_STAGED_TC_PTR, WINO_PATH_STAGED_DP4A) implement it: a
+ * plan on another path moves to the staged tcgen05 path (or the staged dp4a path), forcing
+ * another path afterwards returns WINO_ERR_UNSUPPORTED, and wino_plan_multipliers keeps
+ * reporting the per-layer values.  Synchronous (one small host-to-device copy);
+ * WINO_ERR_INVALID for a bad scale, WINO_ERR_CUDA without a device. */
 int wino_plan_set_channel_scales(wino_plan_t* plan, const float* s_w_K, const float* s_U_K,
-                                 const float* s_Y_K);
+                                 const float* s_M_K, const float* s_Y_K);
 
 /* The five fixed multipliers the plan uses, for inspection:
  * out[0]=s_x/s_V, out[1]=s_w/s_U, out[2]=s_U*s_V/s_M, out[3]=s_acc/s_Y, out[4]=s_acc. */

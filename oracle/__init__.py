@@ -53,7 +53,8 @@ class DescC(ct.Structure):
                 ("BT", ct.c_void_p), ("G", ct.c_void_p), ("AT", ct.c_void_p),
                 ("q_x", QuantC), ("q_w", QuantC), ("q_V", QuantC), ("q_U", QuantC),
                 ("q_M", QuantC), ("q_Y", QuantC), ("out_dtype", ct.c_int32),
-                ("s_w_K", ct.c_void_p), ("s_U_K", ct.c_void_p), ("s_Y_K", ct.c_void_p)]
+                ("s_w_K", ct.c_void_p), ("s_U_K", ct.c_void_p), ("s_M_K", ct.c_void_p),
+                ("s_Y_K", ct.c_void_p)]
 
 
 @dataclass
@@ -88,9 +89,10 @@ class Layer:
     q_M: Quant = field(default_factory=Quant)
     q_Y: Quant = field(default_factory=Quant)
     out_dtype: int = 0
-    # per-output-channel scales (K floats) replacing q_w.scale / q_U.scale / q_Y.scale
+    # per-output-channel scales (K floats) replacing q_w.scale / q_U.scale / q_M.scale / q_Y.scale
     s_w_K: Optional[np.ndarray] = None
     s_U_K: Optional[np.ndarray] = None
+    s_M_K: Optional[np.ndarray] = None
     s_Y_K: Optional[np.ndarray] = None
 
     @property
@@ -141,14 +143,15 @@ class _Keep:
         t = L.t
         assert self.BT.shape == (t, t) and self.G.shape == (t, 3) and self.AT.shape == (L.m, t)
         self.per_K = []
-        for a in (L.s_w_K, L.s_U_K, L.s_Y_K):
+        for a in (L.s_w_K, L.s_U_K, L.s_M_K, L.s_Y_K):
             if a is not None:
                 a = _f32(a)
                 assert a.shape == (L.K,) and np.all(a > 0)
             self.per_K.append(a)
         self.d = DescC(L.N, L.C, L.H, L.W, L.K, L.m, _p(self.BT), _p(self.G), _p(self.AT),
                        L.q_x.c(), L.q_w.c(), L.q_V.c(), L.q_U.c(), L.q_M.c(), L.q_Y.c(),
-                       L.out_dtype, _p(self.per_K[0]), _p(self.per_K[1]), _p(self.per_K[2]))
+                       L.out_dtype, _p(self.per_K[0]), _p(self.per_K[1]), _p(self.per_K[2]),
+                       _p(self.per_K[3]))
 
     @property
     def ref(self):

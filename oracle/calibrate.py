@@ -42,3 +42,38 @@ def calibrate(L: Layer, x_q, w_q, bias=None) -> Layer:
     yf = output_stage(Lf, M, mq, bias)
     L.q_Y.scale = _scale(float(np.max(np.abs(yf))))
     return L
+
+
+def calibrate_per_channel(L: Layer, x_q, w_q, bias=None, output_per_channel: bool = False) -> Layer:
+    """Per-output-channel variant (Section 7): L.s_w_K must be set (the scales the filters in
+    w_q were quantized with); fills q_V, s_U_K (max-abs of each transformed filter), s_M_K
+    (max-abs of each channel's Hadamard sums) and q_Y (one scale: the next layer sums over
+    these channels), or s_Y_K when ``output_per_channel``."""
+    assert L.s_w_K is not None
+    L = copy.deepcopy(L)
+    L.s_U_K = None
+    L.s_M_K = None
+    L.s_Y_K = None
+    s_w = np.asarray(L.s_w_K, np.float32).astype(np.float64)
+    _, Vf = input_stage(L, x_q, want_f32=True)
+    L.q_V.scale = _scale(float(np.max(np.abs(Vf))) * float(np.float32(L.q_x.scale)))
+    _, Uf = weight_stage(L, w_q, want_f32=True)                  # [t*t][K][C], code units
+    u_max = np.max(np.abs(Uf.astype(np.float64)), axis=(0, 2)) * s_w
+    L.s_U_K = np.array([_scale(v) for v in u_max], np.float32)
+    Vq = input_stage(L, x_q)
+    Uq = weight_stage(L, w_q)
+    M = hadamard(L, Vq, Uq)
+    sUV = L.s_U_K.astype(np.float64) * float(np.float32(L.q_V.scale))
+    if L.q_M.enabled:
+        L.s_M_K = np.array([_scale(v) for v in np.abs(M).max(axis=(0, 1)) * sUV], np.float32)
+        mq = quantize_M(L, M)
+    else:
+        mq = None
+    Lf = copy.deepcopy(L)
+    Lf.out_dtype = 1
+    yf = output_stage(Lf, M, mq, bias)
+    if output_per_channel:
+        L.s_Y_K = np.array([_scale(v) for v in np.abs(yf).max(axis=(0, 1, 2))], np.float32)
+    else:
+        L.q_Y.scale = _scale(float(np.max(np.abs(yf))))
+    return L

@@ -165,11 +165,14 @@ struct Desc {
   int32_t out_dtype;  // 0 = int8, 1 = float
   // Per-output-channel scales (Section 7 names per-channel quantization as the next
   // step beyond the per-layer scales of Section 5.1): K floats each, or null for the
-  // per-layer scale of q_w / q_U / q_Y.  Zero points and code ranges stay per layer.
-  const float *s_w_K, *s_U_K, *s_Y_K;
+  // per-layer scale of q_w / q_U / q_M / q_Y: the four tensors that carry the output-channel
+  // axis (the input side is summed over its channels by the Hadamard stage and keeps one
+  // scale).  Zero points and code ranges stay per layer.
+  const float *s_w_K, *s_U_K, *s_M_K, *s_Y_K;
 };
 inline double scale_w(const Desc& d, int k) { return d.s_w_K ? (double)d.s_w_K[k] : (double)d.q_w.scale; }
 inline double scale_U(const Desc& d, int k) { return d.s_U_K ? (double)d.s_U_K[k] : (double)d.q_U.scale; }
+inline double scale_M(const Desc& d, int k) { return d.s_M_K ? (double)d.s_M_K[k] : (double)d.q_M.scale; }
 inline double scale_Y(const Desc& d, int k) { return d.s_Y_K ? (double)d.s_Y_K[k] : (double)d.q_Y.scale; }
 
 struct Geo {
@@ -267,7 +270,7 @@ int32_t orc_quantize(float v, float mult, int32_t z, int32_t qmin, int32_t qmax)
 // out[0] = s_x/s_V, out[1] = s_w/s_U, out[2] = s_U*s_V/s_M,
 // out[3] = s_acc/s_Y, out[4] = s_acc, where s_acc = s_M when Q_M is enabled and
 // s_U*s_V otherwise.  Per-layer scales only (per-channel scales, when given, replace
-// s_w, s_U and s_Y by their channel's value in the same formulas).
+// s_w, s_U, s_M and s_Y by their channel's value in the same formulas).
 void orc_multipliers(const orc_desc_t* d, float* out) {
   double sUV = (double)d->q_U.scale * (double)d->q_V.scale;
   double s_acc = d->q_M.enabled ? (double)d->q_M.scale : sUV;
@@ -375,7 +378,7 @@ int orc_quantize_M(const orc_desc_t* d, const int32_t* M, int8_t* m_q) {
   const long total = (long)g.t * g.t * g.T * d->K;
   std::vector<float> mult_M((size_t)d->K);   // the accumulator of channel k carries s_U[k] * s_V
   for (int k = 0; k < d->K; ++k)
-    mult_M[k] = ratio_f32(scale_U(*d, k) * (double)d->q_V.scale, d->q_M.scale);
+    mult_M[k] = ratio_f32(scale_U(*d, k) * (double)d->q_V.scale, scale_M(*d, k));
 #pragma omp parallel for schedule(static)
   for (long i = 0; i < total; ++i)
     m_q[i] = (int8_t)quantize((float)M[i], mult_M[i % d->K], d->q_M.zero_point, d->q_M.qmin,
@@ -392,12 +395,12 @@ int orc_output_stage(const orc_desc_t* d, const int32_t* M, const int8_t* m_q,
                      const float* bias, float* Y_f32, void* y) {
   Geo g(*d);
   const int t = g.t, m = g.m, K = d->K, H = d->H, W = d->W;
-  // per output channel: s_acc = s_M when Q_M is enabled and s_U[k] * s_V otherwise;
+  // per output channel: s_acc = s_M[k] when Q_M is enabled and s_U[k] * s_V otherwise;
   // mult_Y = s_acc / s_Y[k]; the bias enters the integer output as bias / s_Y[k]
   std::vector<float> mult_Y_k((size_t)K), s_acc_k((size_t)K), bias_k((size_t)K);
   for (int k = 0; k < K; ++k) {
     const double s_acc_d =
-        d->q_M.enabled ? (double)d->q_M.scale : scale_U(*d, k) * (double)d->q_V.scale;
+        d->q_M.enabled ? scale_M(*d, k) : scale_U(*d, k) * (double)d->q_V.scale;
     mult_Y_k[k] = ratio_f32(s_acc_d, scale_Y(*d, k));
     s_acc_k[k] = (float)s_acc_d;
     bias_k[k] = bias ? (float)((double)bias[k] / scale_Y(*d, k)) : 0.0f;

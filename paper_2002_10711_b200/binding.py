@@ -75,7 +75,7 @@ def _load() -> ct.CDLL:
     lib.wino_workspace_bytes.restype = sz
     lib.wino_plan_path.argtypes = [vp]
     lib.wino_plan_force_path.argtypes = [vp, i32]
-    lib.wino_plan_set_channel_scales.argtypes = [vp, vp, vp, vp]
+    lib.wino_plan_set_channel_scales.argtypes = [vp, vp, vp, vp, vp]
     lib.wino_plan_multipliers.argtypes = [vp, vp]
     lib.wino_transform_weights.argtypes = [vp, vp, vp, vp, vp]
     lib.wino_conv_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -178,10 +178,10 @@ class Plan:
     @classmethod
     def from_layer(cls, L, **kw):
         """L: any object with fields N,C,H,W,K,m,BT,G,AT,q_x..q_Y,out_dtype and, optionally,
-        per-output-channel scales s_w_K, s_U_K, s_Y_K."""
+        per-output-channel scales s_w_K, s_U_K, s_M_K, s_Y_K."""
         plan = cls(L.N, L.C, L.H, L.W, L.K, L.m, L.BT, L.G, L.AT, L.q_x, L.q_w, L.q_V, L.q_U,
                    L.q_M, L.q_Y, out_dtype=L.out_dtype, **kw)
-        per_K = [getattr(L, n, None) for n in ("s_w_K", "s_U_K", "s_Y_K")]
+        per_K = [getattr(L, n, None) for n in ("s_w_K", "s_U_K", "s_M_K", "s_Y_K")]
         if any(a is not None for a in per_K):
             plan.set_channel_scales(*per_K)
         return plan
@@ -208,9 +208,9 @@ class Plan:
     def force_path(self, path: int) -> None:
         _check(_lib.wino_plan_force_path(self._h, path), "wino_plan_force_path")
 
-    def set_channel_scales(self, s_w_K=None, s_U_K=None, s_Y_K=None) -> None:
+    def set_channel_scales(self, s_w_K=None, s_U_K=None, s_M_K=None, s_Y_K=None) -> None:
         """Per-output-channel scales (K floats each; None keeps the per-layer scale)."""
-        keep = [None if a is None else np.ascontiguousarray(a, np.float32) for a in (s_w_K, s_U_K, s_Y_K)]
+        keep = [None if a is None else np.ascontiguousarray(a, np.float32) for a in (s_w_K, s_U_K, s_M_K, s_Y_K)]
         for a in keep:
             if a is not None and a.shape != (self.K,):
                 raise ValueError("channel scales must have shape (K,)")

@@ -25,8 +25,8 @@ struct Params {
   int out_dtype;               // 0 int8, 1 float
 };
 // Per-output-channel scales travel beside Params as a device array `chan` [5][K] (null: the
-// per-layer values of Params): row kChMultU = s_w[k]/s_U[k], kChMultM = s_U[k]*s_V/s_M,
-// kChMultY = s_acc[k]/s_Y[k], kChSAcc = s_acc[k] (s_M with Q_M, else s_U[k]*s_V),
+// per-layer values of Params): row kChMultU = s_w[k]/s_U[k], kChMultM = s_U[k]*s_V/s_M[k],
+// kChMultY = s_acc[k]/s_Y[k], kChSAcc = s_acc[k] (s_M[k] with Q_M, else s_U[k]*s_V),
 // kChSY = s_Y[k].
 enum { kChMultU = 0, kChMultM = 1, kChMultY = 2, kChSAcc = 3, kChSY = 4 };
 

@@ -548,15 +548,15 @@ int wino_plan_force_path(wino_plan_t* pl, int path) {
 }
 
 int wino_plan_set_channel_scales(wino_plan_t* pl, const float* s_w_K, const float* s_U_K,
-                                 const float* s_Y_K) {
+                                 const float* s_M_K, const float* s_Y_K) {
   if (pl == nullptr) return WINO_ERR_INVALID;
   const int K = pl->d.K;
-  if (s_w_K == nullptr && s_U_K == nullptr && s_Y_K == nullptr) {   // back to per-layer scales
+  if (s_w_K == nullptr && s_U_K == nullptr && s_M_K == nullptr && s_Y_K == nullptr) {   // per-layer scales again
     if (pl->chan_dev) cudaFree(pl->chan_dev);
     pl->chan_dev = nullptr;
     return WINO_OK;
   }
-  for (const float* a : {s_w_K, s_U_K, s_Y_K})
+  for (const float* a : {s_w_K, s_U_K, s_M_K, s_Y_K})
     if (a != nullptr)
       for (int k = 0; k < K; ++k)
         if (!std::isfinite(a[k]) || !(a[k] > 0.0f)) return WINO_ERR_INVALID;
@@ -567,10 +567,11 @@ int wino_plan_set_channel_scales(wino_plan_t* pl, const float* s_w_K, const floa
     const double s_w = s_w_K ? (double)s_w_K[k] : (double)d.q_w.scale;
     const double s_U = s_U_K ? (double)s_U_K[k] : (double)d.q_U.scale;
     const double s_Y = s_Y_K ? (double)s_Y_K[k] : (double)d.q_Y.scale;
+    const double s_M = s_M_K ? (double)s_M_K[k] : (double)d.q_M.scale;
     const double sUV = s_U * (double)d.q_V.scale;
-    const double s_acc = d.q_M.enabled ? (double)d.q_M.scale : sUV;
+    const double s_acc = d.q_M.enabled ? s_M : sUV;
     tab[(size_t)kChMultU * K + k] = (float)(s_w / s_U);
-    tab[(size_t)kChMultM * K + k] = d.q_M.enabled ? (float)(sUV / (double)d.q_M.scale) : 1.0f;
+    tab[(size_t)kChMultM * K + k] = d.q_M.enabled ? (float)(sUV / s_M) : 1.0f;
     tab[(size_t)kChMultY * K + k] = (float)(s_acc / s_Y);
     tab[(size_t)kChSAcc * K + k] = (float)s_acc;
     tab[(size_t)kChSY * K + k] = (float)s_Y;

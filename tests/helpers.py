@@ -44,12 +44,13 @@ def build_layer(wl: wi.Workload, N: int | None = None, q_M: bool = True, out_dty
 
 
 def per_channel(L: Layer, seed: int, spread: float = 2.0) -> Layer:
-    """Copy of L whose weight, transformed-weight and output scales vary per output channel
+    """Copy of L whose weight, transformed-weight, Hadamard-sum and output scales vary per output channel
     (the per-layer scale times a seeded factor in [1/spread, spread])."""
-    f_w, f_U, f_Y = wi.channel_factors(seed, L.K, spread)
+    f_w, f_U, f_M, f_Y = wi.channel_factors(seed, L.K, spread)
     P = copy.deepcopy(L)
     P.s_w_K = (np.float32(L.q_w.scale) * f_w).astype(np.float32)
     P.s_U_K = (np.float32(L.q_U.scale) * f_U).astype(np.float32)
+    P.s_M_K = (np.float32(L.q_M.scale) * f_M).astype(np.float32) if L.q_M.enabled else None
     P.s_Y_K = (np.float32(L.q_Y.scale) * f_Y).astype(np.float32)
     return P
 

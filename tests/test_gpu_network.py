@@ -57,11 +57,12 @@ def _run_chain(batch, per_channel_weights=False):
         L.q_Y = Quant(qmin=0)
         L = calibrate(L, x_ref, w_q, None)
         if per_channel_weights:
-            # weights and transformed weights scaled per output channel, activations per
+            # weights, transformed weights and Hadamard sums scaled per output channel, activations per
             # layer (the next layer sums over these channels, so its input has one scale)
-            f_w, f_U, _ = wi.channel_factors(seed + spec["index"], spec["K"], 1.5)
+            f_w, f_U, f_M, _ = wi.channel_factors(seed + spec["index"], spec["K"], 1.5)
             L.s_w_K = (np.float32(L.q_w.scale) * f_w).astype(np.float32)
             L.s_U_K = (np.float32(L.q_U.scale) * f_U).astype(np.float32)
+            L.s_M_K = (np.float32(L.q_M.scale) * f_M).astype(np.float32)
         y_ref = oracle.forward(L, x_ref, w_q)
         g1 = gpu_run(L, x_ref, w_q, None)
         assert (g1["y"] == y_ref).all(), f"layer {spec['index']} (oracle-fed) differs"

@@ -262,12 +262,12 @@ def test_per_channel_scales_move_single_kernel_plans_to_a_staged_path():
     plan = binding.Plan.from_layer(L)
     assert plan.path == FUSED
     P = per_channel(L, 5)
-    plan.set_channel_scales(P.s_w_K, P.s_U_K, P.s_Y_K)
+    plan.set_channel_scales(P.s_w_K, P.s_U_K, P.s_M_K, P.s_Y_K)
     assert plan.path == TC
     for refused in (FUSED, SMALLC, TC_MMA, LAYER):
         with pytest.raises(binding.WinoError):
             plan.force_path(refused)
-    plan.set_channel_scales(None, None, None)       # back to per-layer scales
+    plan.set_channel_scales(None, None, None, None)       # back to per-layer scales
     plan.force_path(FUSED)
     with pytest.raises(binding.WinoError):
         plan.set_channel_scales(np.zeros(L.K, np.float32), None, None)
@@ -279,11 +279,14 @@ def test_only_some_channel_scales_given():
     wl = wi.Workload("pcs", 4300, 2, 32, 6, 6, 32, 4)
     L, x_q, w_q, bias = build_layer(wl)
     P = per_channel(L, 9)
-    P.s_U_K = None                                  # weights and output per channel, U per layer
+    P.s_U_K = None; P.s_M_K = None                  # weights and output per channel, U and M per layer
     _compare(P, x_q, w_q, bias, TC)
     P = per_channel(L, 10)
     P.s_w_K = None; P.s_Y_K = None
     _compare(P, x_q, w_q, bias, DP4A)
+    P = per_channel(L, 11)
+    P.s_w_K = None; P.s_U_K = None; P.s_Y_K = None  # only the Hadamard sums per channel
+    _compare(P, x_q, w_q, bias, TC_PTR)
 
 
 @pytest.mark.parametrize("path", [TC, TC_PTR, DP4A])

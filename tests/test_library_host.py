@@ -132,14 +132,15 @@ def test_channel_scales_are_validated_on_the_host():
     nan = ok.copy(); nan[3] = np.nan
     lib = binding._lib
     for arr in (bad, nan, -ok):
-        assert lib.wino_plan_set_channel_scales(p._h, arr.ctypes.data, None, None) == binding.ERR_INVALID
-        assert lib.wino_plan_set_channel_scales(p._h, None, None, arr.ctypes.data) == binding.ERR_INVALID
+        assert lib.wino_plan_set_channel_scales(p._h, arr.ctypes.data, None, None, None) == binding.ERR_INVALID
+        assert lib.wino_plan_set_channel_scales(p._h, None, None, arr.ctypes.data, None) == binding.ERR_INVALID
+        assert lib.wino_plan_set_channel_scales(p._h, None, None, None, arr.ctypes.data) == binding.ERR_INVALID
     before = p.path
-    assert lib.wino_plan_set_channel_scales(p._h, None, None, None) == binding.WINO_OK   # nothing to undo
+    assert lib.wino_plan_set_channel_scales(p._h, None, None, None, None) == binding.WINO_OK   # nothing to undo
     assert p.path == before
     with pytest.raises(ValueError):
         p.set_channel_scales(np.ones(3, np.float32))
-    rc = lib.wino_plan_set_channel_scales(p._h, ok.ctypes.data, None, None)
+    rc = lib.wino_plan_set_channel_scales(p._h, ok.ctypes.data, None, None, None)
     assert rc in (binding.WINO_OK, binding.ERR_CUDA)      # needs a device for its table
     if rc == binding.WINO_OK:
         assert p.path == binding.PATH_STAGED_TC

@@ -24,6 +24,7 @@ def test_equal_channel_scales_reduce_to_the_per_layer_pipeline(m):
     P = copy.deepcopy(L)
     P.s_w_K = np.full(L.K, L.q_w.scale, np.float32)
     P.s_U_K = np.full(L.K, L.q_U.scale, np.float32)
+    P.s_M_K = np.full(L.K, L.q_M.scale, np.float32)
     P.s_Y_K = np.full(L.K, L.q_Y.scale, np.float32)
     y0, d0 = oracle.forward(L, x_q, w_q, bias=bias, dumps=True)
     y1, d1 = oracle.forward(P, x_q, w_q, bias=bias, dumps=True)
@@ -47,6 +48,8 @@ def test_each_channel_equals_the_per_layer_pipeline_on_that_channel(m, variant):
         S.K = 1
         S.q_w.scale = float(P.s_w_K[k])
         S.q_U.scale = float(P.s_U_K[k])
+        if q_M:
+            S.q_M.scale = float(P.s_M_K[k])
         S.q_Y.scale = float(P.s_Y_K[k])
         yk, dk = oracle.forward(S, x_q, w_q[k:k + 1], bias=bias[k:k + 1], dumps=True)
         assert (d["U_q"][:, k] == dk["U_q"][:, 0]).all()
@@ -70,18 +73,64 @@ def test_stage_functions_follow_the_channel_scales_too():
     assert (oracle.output_stage(P, M, mq, bias) == y).all()
 
 
-def test_power_of_two_rescaling_of_one_channel_leaves_its_codes_unchanged():
-    """Without Q_M, multiplying s_w[k], s_U[k], s_Y[k] and bias[k] by 2^j rescales channel k's
-    real values exactly, so every code of the layer stays what it was."""
-    L, x_q, w_q, bias = _layer(4, 960, q_M=False)
+@pytest.mark.parametrize("q_M", [False, True])
+def test_power_of_two_rescaling_of_one_channel_leaves_its_codes_unchanged(q_M):
+    """Multiplying every scale of channel k (s_w, s_U, s_M, s_Y) and bias[k] by 2^j rescales
+    channel k's real values exactly, so every code of the layer stays what it was."""
+    L, x_q, w_q, bias = _layer(4, 960, q_M=q_M)
     P = per_channel(L, 6)
     Q = copy.deepcopy(P)
-    Q.s_w_K = P.s_w_K.copy(); Q.s_U_K = P.s_U_K.copy(); Q.s_Y_K = P.s_Y_K.copy()
     b2 = bias.copy()
     for k, j in ((1, 3), (3, -2)):
-        Q.s_w_K[k] *= 2.0 ** j; Q.s_U_K[k] *= 2.0 ** j; Q.s_Y_K[k] *= 2.0 ** j
+        for name in ("s_w_K", "s_U_K", "s_M_K", "s_Y_K"):
+            if getattr(Q, name) is not None:
+                getattr(Q, name)[k] *= 2.0 ** j
         b2[k] *= 2.0 ** j
     y0, d0 = oracle.forward(P, x_q, w_q, bias=bias, dumps=True)
     y1, d1 = oracle.forward(Q, x_q, w_q, bias=b2, dumps=True)
     assert (d0["U_q"] == d1["U_q"]).all() and (d0["M"] == d1["M"]).all()
+    assert (d0["m_q"] == d1["m_q"]).all()
     assert (y0 == y1).all()
+
+
+def test_channel_scales_recover_filters_of_small_norm():
+    """What per-channel scales are for (Section 7): filters whose norms differ.  Real weights
+    with gains spread over a factor of 64 are quantized once with one scale and once with one
+    scale per filter; against the double-precision convolution of the real tensors, the
+    low-gain channels come out several times more accurate with per-channel scales, and the
+    high-gain ones no worse."""
+    from helpers import matrices
+    from oracle import Layer, Quant
+    from oracle.calibrate import calibrate, calibrate_per_channel
+    m, N, C, H, W, K = 2, 2, 16, 8, 8, 12
+    x_q = wi.halfnormal_codes(321, wi.S_X, (N, H, W, C))
+    s_x = np.float32(1.0 / 32.0)
+    gains = np.float64(2.0) ** (-(np.arange(K) % 7))              # 1 ... 1/64
+    w_real = wi.normal(321, wi.S_W, K * 9 * C).reshape(K, 3, 3, C) * 0.05 * gains[:, None, None, None]
+    BT, G, AT = matrices(m)
+    ref = oracle.direct_f64(x_q.astype(np.float64) * float(s_x), w_real, pad=1)[0]
+
+    def rel_err(y, ks):
+        return float(np.sqrt(np.mean((y[..., ks] - ref[..., ks]) ** 2) / np.mean(ref[..., ks] ** 2)))
+
+    base = Layer(N, C, H, W, K, m, BT, G, AT, out_dtype=1)
+    base.q_x = Quant(scale=float(s_x))
+    # one scale for all filters
+    s_w = np.float32(np.abs(w_real).max() / 127.0)
+    w_q1 = np.clip(np.rint(w_real / np.float64(s_w)), -127, 127).astype(np.int8)
+    L1 = copy.deepcopy(base)
+    L1.q_w = Quant(scale=float(s_w))
+    L1 = calibrate(L1, x_q, w_q1)
+    y1 = oracle.forward(L1, x_q, w_q1)
+    # one scale per filter
+    s_wk = (np.abs(w_real).max(axis=(1, 2, 3)) / 127.0).astype(np.float32)
+    w_q2 = np.clip(np.rint(w_real / s_wk.astype(np.float64)[:, None, None, None]), -127, 127).astype(np.int8)
+    L2 = copy.deepcopy(base)
+    L2.s_w_K = s_wk
+    L2 = calibrate_per_channel(L2, x_q, w_q2, output_per_channel=True)
+    y2 = oracle.forward(L2, x_q, w_q2)
+    low = [k for k in range(K) if gains[k] <= 1.0 / 16]
+    high = [k for k in range(K) if gains[k] == 1.0]
+    assert rel_err(y1, low) > 4 * rel_err(y2, low), (rel_err(y1, low), rel_err(y2, low))
+    assert rel_err(y2, high) < 1.5 * rel_err(y1, high) + 1e-3
+    assert rel_err(y2, list(range(K))) < 0.05

@@ -97,10 +97,11 @@ def flex_perturb(mat32: np.ndarray, seed: int, stream: int, sigma: float = 0.01)
 
 
 def channel_factors(seed: int, K: int, spread: float = 2.0):
-    """Three arrays of K factors, log-uniform in [1/spread, spread]: what per-output-channel
-    scales for the weights, the transformed weights and the output are multiplied by."""
+    """Four arrays of K factors, log-uniform in [1/spread, spread]: what per-output-channel
+    scales for the weights, the transformed weights, the Hadamard sums and the output are
+    multiplied by."""
     out = []
-    for j in range(3):
+    for j in range(4):
         u = uniform(seed, S_CH + j, K)
         out.append(np.exp((2.0 * u - 1.0) * np.log(spread)).astype(np.float32))
     return out
@@ -114,7 +115,7 @@ POINTS = {
 
 # stream ids
 S_X, S_W, S_BIAS, S_BT, S_G, S_AT, S_M = 1, 2, 3, 4, 5, 6, 7
-S_CH = 8   # per-output-channel scale factors (three consecutive streams)
+S_CH = 8   # per-output-channel scale factors (four consecutive streams)
 
 
 @dataclass(frozen=True)
