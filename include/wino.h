@@ -176,6 +176,13 @@ int wino_plan_multipliers(const wino_plan_t* plan, float out[5]);
 int wino_transform_weights(wino_plan_t* plan, const int8_t* w_KRSC_dev, int8_t* Uq_dev,
                            uint32_t* absmax_dev, void* stream);
 
+/* The same transform, recording max |U| of every filter (before quantization, in units of
+ * the weight codes) in absmax_K_dev[k] as float bits (device, uint32[K], caller-zeroed): the
+ * statistic a per-output-channel scale for the transformed weights is set from (see
+ * wino_plan_set_channel_scales).  Uq_dev is written as by wino_transform_weights. */
+int wino_transform_weights_channel_stats(wino_plan_t* plan, const int8_t* w_KRSC_dev,
+                                         int8_t* Uq_dev, uint32_t* absmax_K_dev, void* stream);
+
 /* The forward pass (paper: Eq. 1 with the quantizers of Fig. 2): input
  * transform, Hadamard stage as t*t int8 GEMMs over channels with int32
  * accumulation, output transform, bias, output quantizer.

@@ -26,7 +26,7 @@ STATIC_SCRATCH_BYTES = 20 * 1024 * 1024
 EXPORTS = [
     "wino_plan", "wino_weight_bytes", "wino_workspace_bytes", "wino_plan_path",
     "wino_plan_force_path", "wino_plan_set_channel_scales", "wino_plan_multipliers",
-    "wino_transform_weights",
+    "wino_transform_weights", "wino_transform_weights_channel_stats",
     "wino_conv_forward", "wino_conv_forward_static", "wino_calibrate_forward",
     "wino_direct_conv_forward", "wino_direct_last_status", "wino_last_status", "wino_debug_dump_stage",
     "wino_debug_forward_accumulators", "wino_debug_run_stages", "wino_debug_mma_probe",
@@ -78,6 +78,7 @@ def _load() -> ct.CDLL:
     lib.wino_plan_set_channel_scales.argtypes = [vp, vp, vp, vp, vp]
     lib.wino_plan_multipliers.argtypes = [vp, vp]
     lib.wino_transform_weights.argtypes = [vp, vp, vp, vp, vp]
+    lib.wino_transform_weights_channel_stats.argtypes = [vp, vp, vp, vp, vp]
     lib.wino_conv_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp]
     lib.wino_conv_forward_static.argtypes = [vp, vp, vp, vp, vp, vp]
     lib.wino_calibrate_forward.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
@@ -230,6 +231,11 @@ class Plan:
     def transform_weights(self, w_dev, Uq_dev, absmax_dev=None, stream=None) -> None:
         _check(_lib.wino_transform_weights(self._h, _dptr(w_dev), _dptr(Uq_dev), _dptr(absmax_dev),
                                            _stream_handle(stream)), "wino_transform_weights")
+
+    def transform_weights_channel_stats(self, w_dev, Uq_dev, absmax_K_dev, stream=None) -> None:
+        _check(_lib.wino_transform_weights_channel_stats(
+            self._h, _dptr(w_dev), _dptr(Uq_dev), _dptr(absmax_K_dev), _stream_handle(stream)),
+            "wino_transform_weights_channel_stats")
 
     def conv_forward(self, x_dev, Uq_dev, bias_dev, y_dev, workspace_dev, stream=None) -> None:
         _check(_lib.wino_conv_forward(self._h, _dptr(x_dev), _dptr(Uq_dev), _dptr(bias_dev),

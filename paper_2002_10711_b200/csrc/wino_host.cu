@@ -609,7 +609,16 @@ int wino_transform_weights(wino_plan_t* pl, const int8_t* w, int8_t* Uq, uint32_
   if (!aligned16(w) || !aligned16(Uq)) return WINO_ERR_ALIGNMENT;
   if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
   pl->launches++;
-  return launch_weight_transform(pl->p, pl->chan_dev, w, Uq, absmax, (cudaStream_t)stream);
+  return launch_weight_transform(pl->p, pl->chan_dev, w, Uq, absmax, nullptr, (cudaStream_t)stream);
+}
+
+int wino_transform_weights_channel_stats(wino_plan_t* pl, const int8_t* w, int8_t* Uq,
+                                         uint32_t* absmax_K, void* stream) {
+  if (pl == nullptr || w == nullptr || Uq == nullptr || absmax_K == nullptr) return WINO_ERR_INVALID;
+  if (!aligned16(w) || !aligned16(Uq)) return WINO_ERR_ALIGNMENT;
+  if (pl->status_dev == nullptr) return WINO_ERR_CUDA;
+  pl->launches++;
+  return launch_weight_transform(pl->p, pl->chan_dev, w, Uq, nullptr, absmax_K, (cudaStream_t)stream);
 }
 
 int wino_conv_forward(wino_plan_t* pl, const int8_t* x, const int8_t* Uq, const float* bias,

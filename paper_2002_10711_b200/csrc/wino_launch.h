@@ -65,8 +65,10 @@ int set_max_smem(DeviceOnce& once, int dev, Kern kernel, size_t smem) {
   });
 }
 
+// absmax (nullable): one word, max |U| of the layer; absmax_K (nullable): K words, max |U| of
+// each filter; both as float bits, caller-zeroed.
 int launch_weight_transform(const Params& p, const float* chan, const int8_t* w, int8_t* Uq,
-                            unsigned* absmax, cudaStream_t st);
+                            unsigned* absmax, unsigned* absmax_K, cudaStream_t st);
 int launch_input_transform(const Params& p, const LaunchOpt& o, const int8_t* x, int8_t* Vq,
                            unsigned* absmax, cudaStream_t st);
 int launch_output_transform(const Params& p, const LaunchOpt& o, float s_Y, const void* mbuf,

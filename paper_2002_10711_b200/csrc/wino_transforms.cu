@@ -5,7 +5,7 @@ namespace wino {
 
 #define WINO_DECL(m)                                                                              \
   int launch_weight_transform_m##m(const Params&, const float*, const int8_t*, int8_t*, unsigned*, \
-                                   cudaStream_t);                                                 \
+                                   unsigned*, cudaStream_t);                                      \
   int launch_input_transform_m##m(const Params&, const LaunchOpt&, const int8_t*, int8_t*,        \
                                   unsigned*, cudaStream_t);                                       \
   int launch_output_transform_m##m(const Params&, const LaunchOpt&, float, const void*,           \
@@ -20,10 +20,10 @@ WINO_DECL(6)
 #undef WINO_DECL
 
 int launch_weight_transform(const Params& p, const float* chan, const int8_t* w, int8_t* Uq,
-                            unsigned* absmax, cudaStream_t st) {
-  return p.m == 2 ? launch_weight_transform_m2(p, chan, w, Uq, absmax, st)
-       : p.m == 4 ? launch_weight_transform_m4(p, chan, w, Uq, absmax, st)
-                  : launch_weight_transform_m6(p, chan, w, Uq, absmax, st);
+                            unsigned* absmax, unsigned* absmax_K, cudaStream_t st) {
+  return p.m == 2 ? launch_weight_transform_m2(p, chan, w, Uq, absmax, absmax_K, st)
+       : p.m == 4 ? launch_weight_transform_m4(p, chan, w, Uq, absmax, absmax_K, st)
+                  : launch_weight_transform_m6(p, chan, w, Uq, absmax, absmax_K, st);
 }
 int launch_input_transform(const Params& p, const LaunchOpt& o, const int8_t* x, int8_t* Vq,
                            unsigned* absmax, cudaStream_t st) {

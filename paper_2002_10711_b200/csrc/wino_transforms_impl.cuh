@@ -32,7 +32,7 @@ template <int M, int CPT>
 __global__ void __launch_bounds__(128)
 k_weight_transform(const __grid_constant__ Params p, const float* __restrict__ chan,
                    const int8_t* __restrict__ w, int8_t* __restrict__ Uq,
-                   unsigned* __restrict__ absmax) {
+                   unsigned* __restrict__ absmax, unsigned* __restrict__ absmax_K) {
   constexpr int T_ = M + 2;
   typedef typename Pack<CPT>::type PT;
   const int CG = p.C / CPT;
@@ -83,6 +83,7 @@ k_weight_transform(const __grid_constant__ Params p, const float* __restrict__ c
     PT* Up = reinterpret_cast<PT*>(Uq);
 #pragma unroll
     for (int xi = 0; xi < T_ * T_; ++xi) Up[((long)xi * p.K + k) * CG + cg] = (PT)out[xi];
+    if (absmax_K != nullptr) atomic_absmax(absmax_K + k, vmax);   // this thread's filter only
   }
   if (absmax != nullptr) atomic_absmax(absmax, vmax);
 }
@@ -273,18 +274,18 @@ int pick_cpt(long items_times_channels) {
 
 template <int M, int CPT>
 int weight_cpt(const Params& p, const float* chan, const int8_t* w, int8_t* Uq, unsigned* absmax,
-               cudaStream_t st) {
+               unsigned* absmax_K, cudaStream_t st) {
   const long total = (long)p.K * (p.C / CPT);
   return launch_kernel(k_weight_transform<M, CPT>, dim3((unsigned)((total + 127) / 128)), dim3(128),
-                       0, st, false, p, chan, w, Uq, absmax);
+                       0, st, false, p, chan, w, Uq, absmax, absmax_K);
 }
 template <int M>
 int weight_m(const Params& p, const float* chan, const int8_t* w, int8_t* Uq, unsigned* absmax,
-             cudaStream_t st) {
+             unsigned* absmax_K, cudaStream_t st) {
   const int cpt = pick_cpt((long)p.K * p.C);
-  return cpt == 4 ? weight_cpt<M, 4>(p, chan, w, Uq, absmax, st)
-       : cpt == 2 ? weight_cpt<M, 2>(p, chan, w, Uq, absmax, st)
-                  : weight_cpt<M, 1>(p, chan, w, Uq, absmax, st);
+  return cpt == 4 ? weight_cpt<M, 4>(p, chan, w, Uq, absmax, absmax_K, st)
+       : cpt == 2 ? weight_cpt<M, 2>(p, chan, w, Uq, absmax, absmax_K, st)
+                  : weight_cpt<M, 1>(p, chan, w, Uq, absmax, absmax_K, st);
 }
 
 template <int M, int MODE, int CPT>
@@ -357,8 +358,9 @@ int output_m(const Params& p, const LaunchOpt& o, float s_Y, const void* mbuf, c
 // Entry points for this translation unit's tile size (one unit per m keeps the
 // build parallel).
 int WINO_CAT(launch_weight_transform_m, WINO_M)(const Params& p, const float* chan, const int8_t* w,
-                                                 int8_t* Uq, unsigned* absmax, cudaStream_t st) {
-  return weight_m<WINO_M>(p, chan, w, Uq, absmax, st);
+                                                 int8_t* Uq, unsigned* absmax, unsigned* absmax_K,
+                                                 cudaStream_t st) {
+  return weight_m<WINO_M>(p, chan, w, Uq, absmax, absmax_K, st);
 }
 int WINO_CAT(launch_input_transform_m, WINO_M)(const Params& p, const LaunchOpt& o,
                                                 const int8_t* x, int8_t* Vq, unsigned* absmax,

@@ -359,6 +359,42 @@ def test_gpu_calibration_matches_oracle_calibration():
         assert tuple(np.float32(got)) == tuple(np.float32(want)), (name, got, want)
 
 
+@pytest.mark.parametrize("m,q_M,per_k_out", [(2, True, False), (4, True, True), (6, False, False)])
+def test_gpu_per_channel_calibration_matches_oracle_calibration(m, q_M, per_k_out):
+    """The library-side per-channel calibration (per-filter statistic of the weight transform,
+    stage dumps) against the oracle's, scale for scale; then the layer under those scales."""
+    import copy
+    from paper_2002_10711_b200 import binding
+    from paper_2002_10711_b200.layer import calibrate_per_channel
+    from oracle.calibrate import calibrate_per_channel as oracle_calibrate
+    wl = wi.Workload("pccal2", 4600 + m, 3, 32, 9, 7, 48, m)
+    L, x_q, w_q, bias = build_layer(wl, q_M=q_M)
+    L.s_w_K = (np.float32(L.q_w.scale) * wi.channel_factors(77, L.K, 3.0)[0]).astype(np.float32)
+    want = oracle_calibrate(L, x_q, w_q, bias, output_per_channel=per_k_out)
+
+    def make_plan(s_V, s_U, s_M, s_Y, out_dtype):
+        L2 = copy.deepcopy(L)
+        L2.s_w_K = None
+        L2.q_V.scale, L2.q_U.scale, L2.q_M.scale, L2.q_Y.scale = s_V, s_U, s_M, s_Y
+        L2.out_dtype = out_dtype
+        return binding.Plan.from_layer(L2)
+
+    s_V, s_U_K, s_M_K, s_Y = calibrate_per_channel(make_plan, x_q, w_q, bias, L.q_x.scale, L.s_w_K,
+                                                   output_per_channel=per_k_out)
+    assert np.float32(s_V) == np.float32(want.q_V.scale)
+    assert (s_U_K.view(np.uint32) == want.s_U_K.view(np.uint32)).all()
+    if q_M:
+        assert (s_M_K.view(np.uint32) == want.s_M_K.view(np.uint32)).all()
+    else:
+        assert s_M_K is None and want.s_M_K is None
+    if per_k_out:
+        assert (s_Y.view(np.uint32) == want.s_Y_K.view(np.uint32)).all()
+    else:
+        assert np.float32(s_Y) == np.float32(want.q_Y.scale)
+    g = _compare(want, x_q, w_q, bias, TC)
+    assert np.abs(g["y"]).max() >= 120          # the calibrated output scale fills the range
+
+
 @pytest.mark.parametrize("path", [TC, DP4A])
 def test_calibration_statistics_with_channel_scales(path):
     """The four max-abs statistics of a calibration pass on a plan with per-channel scales,
