@@ -295,12 +295,21 @@ def direct_conv_i32(x_q, w_q, z_x=0, z_w=0, stride=1) -> np.ndarray:
     return acc
 
 
-def requantize_acc(acc, s_in: float, q_Y: Quant, bias=None) -> np.ndarray:
+def requantize_acc(acc, s_in: float, q_Y: Quant, bias=None, s_in_K=None, s_Y_K=None) -> np.ndarray:
+    """Output quantizer on direct-convolution accumulators; s_in_K (float64, the exact products
+    s_x * s_w[k]) and s_Y_K (float32) give per-output-channel scales."""
     acc = np.ascontiguousarray(acc, np.int32)
     K = acc.shape[-1]
     bias = None if bias is None else _f32(bias)
     y = np.zeros(acc.shape, np.int8)
     qc = q_Y.c()
+    if s_in_K is not None or s_Y_K is not None:
+        s_in_K = None if s_in_K is None else np.ascontiguousarray(s_in_K, np.float64)
+        s_Y_K = None if s_Y_K is None else _f32(s_Y_K)
+        assert (s_in_K is None or s_in_K.shape == (K,)) and (s_Y_K is None or s_Y_K.shape == (K,))
+        lib().orc_requantize_acc_channels(ct.c_long(acc.size), K, _p(acc), ct.c_double(s_in), _p(s_in_K),
+                                          _p(bias), ct.byref(qc), _p(s_Y_K), _p(y))
+        return y
     lib().orc_requantize_acc(ct.c_long(acc.size), K, _p(acc), ct.c_double(s_in), _p(bias),
                              ct.byref(qc), _p(y))
     return y

@@ -522,6 +522,24 @@ int orc_requantize_acc(long count, int K, const int32_t* acc, double s_in, const
   return 0;
 }
 
+// The same with per-output-channel scales (Section 7): s_in_K[k] (nullable) replaces s_in
+// and s_Y_K[k] (nullable) replaces q_Y->scale for channel k.
+int orc_requantize_acc_channels(long count, int K, const int32_t* acc, double s_in,
+                                const double* s_in_K, const float* bias, const orc_quant_t* q_Y,
+                                const float* s_Y_K, int8_t* y) {
+#pragma omp parallel for schedule(static)
+  for (long i = 0; i < count; ++i) {
+    int k = (int)(i % K);
+    const double s_in_k = s_in_K ? s_in_K[k] : s_in;
+    const double s_Y_k = s_Y_K ? (double)s_Y_K[k] : (double)q_Y->scale;
+    const float mult = (float)(s_in_k / s_Y_k);
+    float bs = bias ? (float)((double)bias[k] / s_Y_k) : 0.0f;
+    float yf = std::fmaf((float)acc[i], mult, bs);
+    y[i] = (int8_t)quantize(yf, 1.0f, q_Y->zero_point, q_Y->qmin, q_Y->qmax);
+  }
+  return 0;
+}
+
 // Un-quantized double-precision Winograd convolution (Eq. 1) and direct
 // convolution on real-valued tensors; pad is 0 ("valid") or 1.  Both return
 // the number of general multiplications they performed per (input channel,

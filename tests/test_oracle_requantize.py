@@ -151,3 +151,31 @@ def test_float_output_whole_tensor_exact(m, q_M):
                     assert Fraction(float(y[n, h, w, k])) == want
                     checked += 1
     assert checked == y.size and np.abs(y).max() > 0
+
+
+def test_per_channel_scales_equal_the_per_layer_quantizer_channel_by_channel():
+    """requantize_acc with per-output-channel scales: every channel must equal the per-layer
+    quantizer (pinned above) applied to that channel with its own scales; equal scales must
+    reproduce the per-layer result."""
+    K = 7
+    acc = ((wi.bits64(71, 5, 6 * 5 * K) % np.uint64(40001)).astype(np.int64) - 20000).astype(np.int32).reshape(6, 5, K)
+    bias = wi.bias_values(71, 3, K, 2.0)
+    s_x = np.float32(1 / 32)
+    f_w, _, _, f_Y = wi.channel_factors(71, K, 4.0)
+    s_w_K = (np.float32(0.003) * f_w).astype(np.float32)
+    s_Y_K = (np.float32(0.02) * f_Y).astype(np.float32)
+    s_in_K = s_w_K.astype(np.float64) * np.float64(s_x)
+    q_Y = Quant(scale=0.02, zero_point=3, qmin=-100, qmax=120)
+    got = oracle.requantize_acc(acc, 0.0, q_Y, bias, s_in_K=s_in_K, s_Y_K=s_Y_K)
+    for k in range(K):
+        q_k = Quant(scale=float(s_Y_K[k]), zero_point=3, qmin=-100, qmax=120)
+        want = oracle.requantize_acc(acc[..., k:k + 1], float(s_in_K[k]), q_k, bias[k:k + 1])
+        assert (got[..., k] == want[..., 0]).all(), k
+    assert len(np.unique(got)) > 20
+    s_in = float(np.float64(s_x) * np.float64(np.float32(0.003)))
+    same = oracle.requantize_acc(acc, s_in, q_Y, bias, s_in_K=np.full(K, s_in), s_Y_K=np.full(K, 0.02, np.float32))
+    assert (same == oracle.requantize_acc(acc, s_in, q_Y, bias)).all()
+    only_w = oracle.requantize_acc(acc, s_in, q_Y, bias, s_in_K=s_in_K)
+    for k in range(K):
+        want = oracle.requantize_acc(acc[..., k:k + 1], float(s_in_K[k]), q_Y, bias[k:k + 1])
+        assert (only_w[..., k] == want[..., 0]).all()
