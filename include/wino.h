@@ -255,6 +255,12 @@ typedef struct {
   int32_t N, C, H, W, K, stride;
   wino_quant_t q_x, q_w, q_Y;
   int32_t out_dtype;
+  /* Per-output-channel scales (paper: Section 7), DEVICE arrays of K positive floats or NULL:
+   * s_w_K_dev[k] replaces q_w.scale for filter k, s_Y_K_dev[k] replaces q_Y.scale for output
+   * channel k.  The kernels form, per channel, (float)((double)s_x * s_w[k] / s_Y[k]) and
+   * (float)((double)bias[k] / s_Y[k]); the values are not validated (they live on the device). */
+  const float* s_w_K_dev;
+  const float* s_Y_K_dev;
 } wino_direct_desc_t;
 int wino_direct_conv_forward(const wino_direct_desc_t* desc, const int8_t* x_NHWC_dev,
                              const int8_t* w_KRSC_dev, const float* bias_K_dev, void* y_dev,

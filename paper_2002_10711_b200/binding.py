@@ -52,7 +52,8 @@ class DescC(ct.Structure):
 class DirectDescC(ct.Structure):
     _fields_ = [("N", ct.c_int32), ("C", ct.c_int32), ("H", ct.c_int32), ("W", ct.c_int32),
                 ("K", ct.c_int32), ("stride", ct.c_int32),
-                ("q_x", QuantC), ("q_w", QuantC), ("q_Y", QuantC), ("out_dtype", ct.c_int32)]
+                ("q_x", QuantC), ("q_w", QuantC), ("q_Y", QuantC), ("out_dtype", ct.c_int32),
+                ("s_w_K_dev", ct.c_void_p), ("s_Y_K_dev", ct.c_void_p)]
 
 
 class WinoError(RuntimeError):
@@ -145,9 +146,12 @@ def direct_last_status(stream=None) -> int:
 
 
 def direct_conv_forward(N, C, H, W, K, stride, q_x, q_w, q_Y, x_dev, w_dev, bias_dev, y_dev,
-                        out_dtype=0, stream=None) -> None:
-    """wino_direct_conv_forward: direct int8 3x3 convolution, stride 1 or 2."""
-    d = DirectDescC(N, C, H, W, K, stride, _quant(q_x), _quant(q_w), _quant(q_Y), out_dtype)
+                        out_dtype=0, stream=None, s_w_K_dev=None, s_Y_K_dev=None) -> None:
+    """wino_direct_conv_forward: direct int8 3x3 convolution, stride 1 or 2; s_w_K_dev and
+    s_Y_K_dev: optional per-output-channel scales (float32 tensors of K elements on the device)."""
+    d = DirectDescC(N, C, H, W, K, stride, _quant(q_x), _quant(q_w), _quant(q_Y), out_dtype,
+                    None if s_w_K_dev is None else s_w_K_dev.data_ptr(),
+                    None if s_Y_K_dev is None else s_Y_K_dev.data_ptr())
     _check(_lib.wino_direct_conv_forward(ct.byref(d), _dptr(x_dev), _dptr(w_dev), _dptr(bias_dev),
                                          _dptr(y_dev), _stream_handle(stream)),
            "wino_direct_conv_forward")

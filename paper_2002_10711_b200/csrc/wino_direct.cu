@@ -12,7 +12,25 @@ struct DirectParams {
   int z_x, z_w, z_Y;
   float mult, s_in, s_Y, lo_Y, hi_Y;
   int out_dtype;
+  // per-output-channel scales (device arrays of K floats, nullable) and the per-layer scales
+  const float* s_w_K;
+  const float* s_Y_K;
+  float s_x, s_w;
 };
+
+// Channel k's output arithmetic: the multiplier on the accumulator (s_x * s_w[k] / s_Y[k] for
+// integer output, s_x * s_w[k] for float output; the product of the two scales is exact in
+// double) and the output scale the bias is divided by.
+__device__ __forceinline__ void channel_scales(const DirectParams& p, int k, float& mult, float& s_in,
+                                               float& s_Y) {
+  mult = p.mult; s_in = p.s_in; s_Y = p.s_Y;
+  if (p.s_w_K != nullptr || p.s_Y_K != nullptr) {
+    const double s_in_k = (double)p.s_x * (double)(p.s_w_K != nullptr ? __ldg(p.s_w_K + k) : p.s_w);
+    if (p.s_Y_K != nullptr) s_Y = __ldg(p.s_Y_K + k);
+    mult = (float)(s_in_k / (double)s_Y);
+    s_in = (float)s_in_k;
+  }
+}
 
 // KPT output channels per thread.  Consecutive lanes take consecutive output
 // pixels, so a weight word is one broadcast load for the warp and every lane
@@ -72,8 +90,10 @@ k_direct_conv(const DirectParams p, const int8_t* __restrict__ x, const int8_t* 
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const int k = kg * KPT + j4 + j;
-        const float b = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)p.s_Y) : 0.0f;
-        const float yf = __fmaf_rn(__int2float_rn(acc[j4 + j]), p.mult, b);
+        float mult, s_in, s_Y;
+        channel_scales(p, k, mult, s_in, s_Y);
+        const float b = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)s_Y) : 0.0f;
+        const float yf = __fmaf_rn(__int2float_rn(acc[j4 + j]), mult, b);
         const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
         word |= ((uint32_t)(magic_to_int(r) + p.z_Y) & 0xFFu) << (8 * j);
       }
@@ -82,7 +102,9 @@ k_direct_conv(const DirectParams p, const int8_t* __restrict__ x, const int8_t* 
 #pragma unroll
       for (int j = 0; j < 4; ++j) {
         const float b = bias != nullptr ? __ldg(bias + kg * KPT + j4 + j) : 0.0f;
-        reinterpret_cast<float*>(y)[o + j4 + j] = __fmaf_rn(__int2float_rn(acc[j4 + j]), p.s_in, b);
+        float mult, s_in, s_Y;
+        channel_scales(p, kg * KPT + j4 + j, mult, s_in, s_Y);
+        reinterpret_cast<float*>(y)[o + j4 + j] = __fmaf_rn(__int2float_rn(acc[j4 + j]), s_in, b);
       }
     }
   }
@@ -116,22 +138,25 @@ k_direct_conv_bytes(const DirectParams p, const int8_t* __restrict__ x, const in
     }
   }
   const long o = (((long)n * p.Ho + ho) * p.Wo + wo) * p.K + k;
+  float mult, s_in, s_Y;
+  channel_scales(p, k, mult, s_in, s_Y);
   if (p.out_dtype == 0) {
-    const float b = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)p.s_Y) : 0.0f;
-    const float yf = __fmaf_rn(__int2float_rn(acc), p.mult, b);
+    const float b = bias != nullptr ? (float)((double)__ldg(bias + k) / (double)s_Y) : 0.0f;
+    const float yf = __fmaf_rn(__int2float_rn(acc), mult, b);
     const float r = __fadd_rn(fminf(fmaxf(yf, p.lo_Y), p.hi_Y), kMagic);
     reinterpret_cast<int8_t*>(y)[o] = (int8_t)(magic_to_int(r) + p.z_Y);
   } else {
     const float b = bias != nullptr ? __ldg(bias + k) : 0.0f;
-    reinterpret_cast<float*>(y)[o] = __fmaf_rn(__int2float_rn(acc), p.s_in, b);
+    reinterpret_cast<float*>(y)[o] = __fmaf_rn(__int2float_rn(acc), s_in, b);
   }
 }
 
 int launch_direct_conv(int N, int C, int H, int W, int K, int stride, int z_x, int z_w, int z_Y,
                        float mult, float s_in, float s_Y, float lo_Y, float hi_Y, int out_dtype,
                        const int8_t* x, const int8_t* w, const float* bias, void* y,
-                       cudaStream_t st) {
+                       const float* s_w_K, const float* s_Y_K, float s_x, float s_w, cudaStream_t st) {
   DirectParams p;
+  p.s_w_K = s_w_K; p.s_Y_K = s_Y_K; p.s_x = s_x; p.s_w = s_w;
   p.N = N; p.C = C; p.H = H; p.W = W; p.K = K; p.stride = stride;
   p.Ho = (H - 1) / stride + 1; p.Wo = (W - 1) / stride + 1;
   p.z_x = z_x; p.z_w = z_w; p.z_Y = z_Y;

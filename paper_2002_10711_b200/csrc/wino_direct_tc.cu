@@ -36,16 +36,18 @@ __device__ __forceinline__ uint64_t desc_sw64(uint32_t smem_addr) {
          (4ull << 61);
 }
 
-__global__ void __launch_bounds__(kDtThreads, 1)
-k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
-                 const DirectTcArgs a, const float* __restrict__ bias, void* __restrict__ y,
-                 int* __restrict__ status) {
+// PK: the weight and output scales vary per output channel (a build of its own: the per-layer
+// kernel keeps its one multiplier in a register).
+template <bool PK>
+__device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, const CUtensorMap& mapW,
+                                                    const DirectTcArgs& a, const float* __restrict__ bias,
+                                                    void* __restrict__ y, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t a_bytes = 128u * (uint32_t)a.cB, b_bytes = (uint32_t)a.BN * (uint32_t)a.cB;
   const uint32_t stage_bytes = a_bytes + b_bytes;
   const uint32_t s_bias = base + (uint32_t)a.stages * stage_bytes;   // K floats
-  const uint32_t bars = s_bias + (uint32_t)a.K * 4u;
+  const uint32_t bars = s_bias + (uint32_t)a.K * (PK ? 8u : 4u);   // PK: K multipliers follow
   const uint32_t bar_full = bars;                           // stages x 8 B
   const uint32_t bar_empty = bar_full + 8u * a.stages;      // stages x 8 B
   const uint32_t bar_acc_full = bar_empty + 8u * a.stages;  // 2 x 8 B
@@ -56,6 +58,8 @@ k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant
   volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
   volatile uint32_t* abort_p = reinterpret_cast<volatile uint32_t*>(gen + (abort_slot - base));
   float* bias_tab = reinterpret_cast<float*>(gen + (s_bias - base));
+  float* mult_tab = bias_tab + a.K;   // PK only
+  (void)mult_tab;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles = a.nW * a.nH * a.nI;
@@ -80,9 +84,16 @@ k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant
   // bias in output-code units (or as it is, for the float output); the bias is a parameter of
   // the layer, not an output of the preceding kernel
   for (int k = threadIdx.x; k < a.K; k += blockDim.x) {
+    float s_Y_k = a.s_Y;
+    if constexpr (PK) {
+      // channel k: accumulator scale s_x * s_w[k] (exact in double), output scale s_Y[k]
+      const double s_in_k = (double)a.s_x * (double)(a.s_w_K != nullptr ? __ldg(a.s_w_K + k) : a.s_w);
+      if (a.s_Y_K != nullptr) s_Y_k = __ldg(a.s_Y_K + k);
+      mult_tab[k] = a.out_dtype == 0 ? (float)(s_in_k / (double)s_Y_k) : (float)s_in_k;
+    }
     float b = 0.0f;
     if (bias != nullptr)
-      b = a.out_dtype == 0 ? (float)((double)__ldg(bias + k) / (double)a.s_Y) : __ldg(bias + k);
+      b = a.out_dtype == 0 ? (float)((double)__ldg(bias + k) / (double)s_Y_k) : __ldg(bias + k);
     bias_tab[k] = b;
   }
   tc_fence_before();
@@ -196,7 +207,8 @@ k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant
             uint32_t word = 0u;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-              const float yf = __fmaf_rn(__int2float_rn((int)acc[4 * q + e]), a.mult, bias_tab[k0 + 4 * q + e]);
+              const float yf = __fmaf_rn(__int2float_rn((int)acc[4 * q + e]),
+                                         PK ? mult_tab[k0 + 4 * q + e] : a.mult, bias_tab[k0 + 4 * q + e]);
               const float rr = __fadd_rn(fminf(fmaxf(yf, lo), hi_c), kMagic);
               word |= ((uint32_t)(magic_to_int(rr) + a.z_Y) & 0xFFu) << (8 * e);
             }
@@ -211,10 +223,10 @@ k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant
 #pragma unroll
           for (int q = 0; q < 8; ++q) {
             float4 v;
-            v.x = __fmaf_rn(__int2float_rn((int)acc[4 * q + 0]), a.s_in, bias_tab[k0 + 4 * q + 0]);
-            v.y = __fmaf_rn(__int2float_rn((int)acc[4 * q + 1]), a.s_in, bias_tab[k0 + 4 * q + 1]);
-            v.z = __fmaf_rn(__int2float_rn((int)acc[4 * q + 2]), a.s_in, bias_tab[k0 + 4 * q + 2]);
-            v.w = __fmaf_rn(__int2float_rn((int)acc[4 * q + 3]), a.s_in, bias_tab[k0 + 4 * q + 3]);
+            v.x = __fmaf_rn(__int2float_rn((int)acc[4 * q + 0]), PK ? mult_tab[k0 + 4 * q + 0] : a.s_in, bias_tab[k0 + 4 * q + 0]);
+            v.y = __fmaf_rn(__int2float_rn((int)acc[4 * q + 1]), PK ? mult_tab[k0 + 4 * q + 1] : a.s_in, bias_tab[k0 + 4 * q + 1]);
+            v.z = __fmaf_rn(__int2float_rn((int)acc[4 * q + 2]), PK ? mult_tab[k0 + 4 * q + 2] : a.s_in, bias_tab[k0 + 4 * q + 2]);
+            v.w = __fmaf_rn(__int2float_rn((int)acc[4 * q + 3]), PK ? mult_tab[k0 + 4 * q + 3] : a.s_in, bias_tab[k0 + 4 * q + 3]);
             dst[q] = v;
           }
         }
@@ -232,6 +244,20 @@ k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant
     tc_fence_after();
     tmem_dealloc(tmem_base, (uint32_t)a.tmem_cols);
   }
+}
+
+__global__ void __launch_bounds__(kDtThreads, 1)
+k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
+                 const DirectTcArgs a, const float* __restrict__ bias, void* __restrict__ y,
+                 int* __restrict__ status) {
+  direct_conv_tc_body<false>(mapX, mapW, a, bias, y, status);
+}
+__global__ void __launch_bounds__(kDtThreads, 1)
+k_direct_conv_tc_per_channel(const __grid_constant__ CUtensorMap mapX,
+                             const __grid_constant__ CUtensorMap mapW, const DirectTcArgs a,
+                             const float* __restrict__ bias, void* __restrict__ y,
+                             int* __restrict__ status) {
+  direct_conv_tc_body<true>(mapX, mapW, a, bias, y, status);
 }
 
 // One status word per device for the plan-less direct convolution.
@@ -292,10 +318,17 @@ int launch_direct_conv_tc(const DirectTcArgs& a, int device, int num_sms, const 
   int* status = direct_tc_status_word(device);
   if (status == nullptr) return -5;
   const size_t stage = (size_t)128 * a.cB + (size_t)a.BN * a.cB;
-  const size_t smem = 1024 + (size_t)a.stages * stage + (size_t)a.K * 4 + 16 * (size_t)a.stages + 64;
+  const bool pk = a.s_w_K != nullptr || a.s_Y_K != nullptr;
+  const size_t smem = 1024 + (size_t)a.stages * stage + (size_t)a.K * (pk ? 8 : 4) + 16 * (size_t)a.stages + 64;
+  const int grid = a.n_items < num_sms ? a.n_items : num_sms;
+  if (pk) {
+    static DeviceOnce once_pk;
+    if (int rc = set_max_smem(once_pk, device, k_direct_conv_tc_per_channel, 227 * 1024)) return rc;
+    return launch_kernel(k_direct_conv_tc_per_channel, dim3((unsigned)grid), dim3(kDtThreads), smem, st,
+                         true, mapX, mapW, a, bias, y, status);
+  }
   static DeviceOnce once;
   if (int rc = set_max_smem(once, device, k_direct_conv_tc, 227 * 1024)) return rc;
-  const int grid = a.n_items < num_sms ? a.n_items : num_sms;
   return launch_kernel(k_direct_conv_tc, dim3((unsigned)grid), dim3(kDtThreads), smem, st, true, mapX, mapW,
                        a, bias, y, status);
 }

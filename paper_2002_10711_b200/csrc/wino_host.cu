@@ -671,6 +671,8 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
   if (!quant_ok(d->q_x) || !quant_ok(d->q_w) || !quant_ok(d->q_Y)) return WINO_ERR_INVALID;
   if (!aligned16(x) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias)))
     return WINO_ERR_ALIGNMENT;
+  if ((reinterpret_cast<uintptr_t>(d->s_w_K_dev) & 3u) != 0 || (reinterpret_cast<uintptr_t>(d->s_Y_K_dev) & 3u) != 0)
+    return WINO_ERR_ALIGNMENT;
   const double s_in = (double)d->q_x.scale * (double)d->q_w.scale;
   if (direct_tc_supported(d->C, d->K, d->H, d->W, d->stride, d->q_x.zero_point, d->q_w.zero_point) &&
       (reinterpret_cast<uintptr_t>(y) & 31u) == 0) {
@@ -684,6 +686,8 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
     a.mult = (float)(s_in / (double)d->q_Y.scale);
     a.s_in = (float)s_in;
     a.s_Y = d->q_Y.scale;
+    a.s_w_K = d->s_w_K_dev; a.s_Y_K = d->s_Y_K_dev;
+    a.s_x = d->q_x.scale; a.s_w = d->q_w.scale;
     a.lo_Y = (float)(d->q_Y.qmin - d->q_Y.zero_point);
     a.hi_Y = (float)(d->q_Y.qmax - d->q_Y.zero_point);
     a.z_Y = d->q_Y.zero_point;
@@ -715,6 +719,7 @@ int wino_direct_conv_forward(const wino_direct_desc_t* d, const int8_t* x, const
                             (float)(s_in / (double)d->q_Y.scale), (float)s_in, d->q_Y.scale,
                             (float)(d->q_Y.qmin - d->q_Y.zero_point),
                             (float)(d->q_Y.qmax - d->q_Y.zero_point), d->out_dtype, x, w, bias, y,
+                            d->s_w_K_dev, d->s_Y_K_dev, d->q_x.scale, d->q_w.scale,
                             (cudaStream_t)stream);
 }
 

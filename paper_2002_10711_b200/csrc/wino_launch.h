@@ -148,16 +148,23 @@ struct DirectTcArgs {
   int n_items;
   float mult, s_in, s_Y, lo_Y, hi_Y;
   int z_Y, out_dtype;
+  // per-output-channel scales (device arrays of K floats, nullable) and the per-layer scales
+  // they replace
+  const float* s_w_K;
+  const float* s_Y_K;
+  float s_x, s_w;
 };
 bool direct_tc_supported(int C, int K, int H, int W, int stride, int z_x, int z_w);
 DirectTcArgs direct_tc_geometry(int N, int C, int H, int W, int K, int stride, int num_sms);
 int* direct_tc_status_word(int device);
 int launch_direct_conv_tc(const DirectTcArgs& a, int device, int num_sms, const CUtensorMap& mapX,
                           const CUtensorMap& mapW, const float* bias, void* y, cudaStream_t st);
+// s_w_K, s_Y_K (nullable device arrays of K floats): per-output-channel scales replacing s_w
+// and s_Y; s_x, s_w: the per-layer scales behind mult and s_in.
 int launch_direct_conv(int N, int C, int H, int W, int K, int stride, int z_x, int z_w, int z_Y,
                        float mult, float s_in, float s_Y, float lo_Y, float hi_Y, int out_dtype,
                        const int8_t* x, const int8_t* w, const float* bias, void* y,
-                       cudaStream_t st);
+                       const float* s_w_K, const float* s_Y_K, float s_x, float s_w, cudaStream_t st);
 
 // Tensor-pipe probe: `iters` back-to-back 128x256x32 int8 MMAs on every SM.
 int launch_mma_peak(int iters, int num_sms, int device, int* status, cudaStream_t st);

@@ -137,3 +137,45 @@ def test_direct_conv_argument_checks():
     with pytest.raises(binding.WinoError) as e:
         binding.direct_conv_forward(1, 8, 8, 8, 16, 1, q, q, q, 16, 24, None, 16, stream=0)   # w not 16-byte aligned
     assert e.value.code == binding.ERR_ALIGNMENT
+
+
+# per-output-channel scales (Section 7) on every direct-convolution kernel: tensor cores
+# (stride 1 and 2), integer dot products, byte-wise
+@pytest.mark.parametrize("shape,stride", [((2, 64, 9, 7, 32), 1), ((3, 128, 8, 8, 64), 2), ((1, 256, 5, 19, 288), 1),
+                                          ((2, 16, 9, 7, 8), 1), ((1, 20, 6, 11, 12), 2), ((2, 3, 16, 16, 6), 1)])
+@pytest.mark.parametrize("which", ["both", "weights_only", "output_only"])
+@pytest.mark.parametrize("out_dtype", [0, 1])
+def test_direct_conv_per_channel_scales(shape, stride, which, out_dtype):
+    import torch
+    from paper_2002_10711_b200 import binding
+    N, C, H, W, K = shape
+    x_q = wi.halfnormal_codes(5600 + C, 1, (N, H, W, C))
+    w_q, s_w = wi.gaussian_weight_codes(5600 + K, 2, (K, 3, 3, C), 0.05)
+    bias = wi.bias_values(5600, 3, K, 0.5)
+    s_x = np.float32(1 / 32)
+    f_w, _, _, f_Y = wi.channel_factors(5600 + K, K, 3.0)
+    acc = oracle.direct_conv_i32(x_q, w_q, stride=stride)
+    s_in = float(np.float64(s_x) * np.float64(s_w))
+    q_Y = Quant(qmin=-120, zero_point=2)
+    q_Y.scale = float(np.float32(max(float(np.abs(acc).max()) * s_in, 1e-6) / 127.0))
+    s_w_K = (np.float32(s_w) * f_w).astype(np.float32) if which != "output_only" else None
+    s_Y_K = (np.float32(q_Y.scale) * f_Y).astype(np.float32) if which != "weights_only" else None
+    s_in_K = None if s_w_K is None else s_w_K.astype(np.float64) * np.float64(s_x)
+    dev = lambda a: None if a is None else torch.from_numpy(a).cuda()
+    Ho, Wo = (H - 1) // stride + 1, (W - 1) // stride + 1
+    y = torch.empty((N, Ho, Wo, K), dtype=torch.float32 if out_dtype else torch.int8, device="cuda")
+    binding.direct_conv_forward(N, C, H, W, K, stride, Quant(scale=float(s_x)), Quant(scale=float(s_w)), q_Y,
+                                dev(x_q), dev(w_q), dev(bias), y, out_dtype=out_dtype,
+                                s_w_K_dev=dev(s_w_K), s_Y_K_dev=dev(s_Y_K))
+    torch.cuda.synchronize()
+    assert binding.direct_last_status() == 0
+    got = y.cpu().numpy()
+    if out_dtype == 0:
+        want = oracle.requantize_acc(acc, s_in, q_Y, bias, s_in_K=s_in_K, s_Y_K=s_Y_K)
+        assert (got == want).all()
+        assert len(np.unique(want)) > 10
+    else:
+        # float output: fmaf(acc, (float)(s_x * s_w[k]), bias[k]), exactly rounded once
+        s_k = (s_in_K if s_in_K is not None else np.full(K, s_in)).astype(np.float32).astype(np.float64)
+        exact = acc.astype(np.float64) * s_k + bias.astype(np.float64)
+        assert (got == exact.astype(np.float32)).all()

@@ -34,7 +34,11 @@ def _run_chain(batch, per_channel_weights=False):
             acc = oracle.direct_conv_i32(x_ref, w_q, stride=2)
             real_max = float(np.abs(acc).max()) * s_x * float(s_w)
             q_Y = Quant(scale=float(np.float32(real_max / 127.0)), qmin=0)
-            x_ref = oracle.requantize_acc(acc, s_x * float(s_w), q_Y)
+            s_w_K = s_in_K = None
+            if per_channel_weights:
+                s_w_K = (np.float32(s_w) * wi.channel_factors(seed + spec["index"], spec["K"], 1.5)[0]).astype(np.float32)
+                s_in_K = s_w_K.astype(np.float64) * np.float64(np.float32(s_x))
+            x_ref = oracle.requantize_acc(acc, s_x * float(s_w), q_Y, s_in_K=s_in_K)
             # the GPU chain runs its strided layers with the library's direct convolution
             import torch
             from paper_2002_10711_b200 import binding
@@ -42,7 +46,8 @@ def _run_chain(batch, per_channel_weights=False):
             wd = torch.from_numpy(w_q).cuda()
             yd = torch.empty(x_ref.shape, dtype=torch.int8, device="cuda")
             binding.direct_conv_forward(batch, spec["C"], spec["H"], spec["W"], spec["K"], 2,
-                                        Quant(scale=s_x), Quant(scale=float(s_w)), q_Y, xd, wd, None, yd)
+                                        Quant(scale=s_x), Quant(scale=float(s_w)), q_Y, xd, wd, None, yd,
+                                        s_w_K_dev=None if s_w_K is None else torch.from_numpy(s_w_K).cuda())
             torch.cuda.synchronize()
             x_gpu = yd.cpu().numpy()
             assert (x_gpu == x_ref).all(), f"layer {spec['index']} (direct, stride 2) differs"
