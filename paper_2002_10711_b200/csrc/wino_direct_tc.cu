@@ -17,6 +17,12 @@
 //
 // For stride 2 (even H and W) the input is addressed as [N][H/2][2][W/2][2*C]: a tap then reads
 // one row parity and one column parity, again a dense box.
+// Narrow layers (one block of output channels, 9 * C * K bytes of weights that fit beside the
+// input ring; the 64- and 128-channel layers of the network): the weights are fetched once per
+// block and stay in shared memory, and the ring's stages carry input boxes only, three taps
+// (one row of the filter) per stage where that fits.  The producer and the MMA warp are
+// single threads of control whose every instruction costs ten to twenty cycles, so what
+// bounds these layers is the number of copies, waits and commits per item, which this halves.
 // Zero points on x or w, odd sizes at stride 2 and channel counts that are not multiples of
 // 64 / 32 stay on the ALU kernel (wino_direct.cu).
 #include "wino_launch.h"
@@ -38,15 +44,18 @@ __device__ __forceinline__ uint64_t desc_sw64(uint32_t smem_addr) {
 
 // PK: the weight and output scales vary per output channel (a build of its own: the per-layer
 // kernel keeps its one multiplier in a register).
-template <bool PK>
+template <bool PK, bool RW>
 __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, const CUtensorMap& mapW,
                                                     const DirectTcArgs& a, const float* __restrict__ bias,
                                                     void* __restrict__ y, int* __restrict__ status) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   const uint32_t a_bytes = 128u * (uint32_t)a.cB, b_bytes = (uint32_t)a.BN * (uint32_t)a.cB;
-  const uint32_t stage_bytes = a_bytes + b_bytes;
-  const uint32_t s_bias = base + (uint32_t)a.stages * stage_bytes;   // K floats
+  // RW: [9 * KB weight slices][stages x taps_per_stage * KB input boxes]; else [stages x (A, B)]
+  const uint32_t res_bytes = RW ? 9u * (uint32_t)a.KB * b_bytes : 0u;
+  const uint32_t stage_bytes = RW ? (uint32_t)(a.taps_per_stage * a.KB) * a_bytes : a_bytes + b_bytes;
+  const uint32_t ring = base + res_bytes;
+  const uint32_t s_bias = ring + (uint32_t)a.stages * stage_bytes;   // K floats
   const uint32_t bars = s_bias + (uint32_t)a.K * (PK ? 8u : 4u);   // PK: K multipliers follow
   const uint32_t bar_full = bars;                           // stages x 8 B
   const uint32_t bar_empty = bar_full + 8u * a.stages;      // stages x 8 B
@@ -54,6 +63,7 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
   const uint32_t bar_acc_empty = bar_acc_full + 16u;        // 2 x 8 B
   const uint32_t tmem_slot = bar_acc_empty + 16u;
   const uint32_t abort_slot = tmem_slot + 4u;
+  const uint32_t bar_w = bar_acc_empty + 32u;               // RW: the resident weights have landed
   uint8_t* gen = smem_raw + (base - smem_u32(smem_raw));
   volatile uint32_t* tmem_slot_p = reinterpret_cast<volatile uint32_t*>(gen + (tmem_slot - base));
   volatile uint32_t* abort_p = reinterpret_cast<volatile uint32_t*>(gen + (abort_slot - base));
@@ -63,7 +73,7 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int n_tiles = a.nW * a.nH * a.nI;
-  const int steps = 9 * a.KB;   // stages per item
+  const int steps = RW ? 9 / a.taps_per_stage : 9 * a.KB;   // stages per item
 
   griddep_launch();
   if (threadIdx.x == 0) {
@@ -75,6 +85,7 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
       mbar_init(bar_acc_full + 8u * b, 1);
       mbar_init(bar_acc_empty + 8u * b, kDtEpiWarps);
     }
+    if (RW) mbar_init(bar_w, 1);
     *abort_p = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     tma_prefetch_map(&mapX);
@@ -109,6 +120,15 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
       // about five hundred: everything that does not change inside an item is computed once per
       // item, and the loops carry running coordinates instead of multiplying)
       const int n_stages = a.stages, kblocks = a.KB, cb = a.cB, strided = a.stride != 1;
+      if constexpr (RW) {
+        // the whole weight tensor, once: slice (tap, channel block) at res + (tap * KB + kb) * b_bytes
+        mbar_expect_tx(bar_w, res_bytes);
+        uint32_t dst = base;
+        for (int tap = 0; tap < 9; ++tap)
+          for (int kb = 0; kb < kblocks; ++kb, dst += b_bytes)
+            tma_load_3d(dst, &mapW, bar_w, kb * cb, tap, 0);
+      }
+      const int tps = RW ? a.taps_per_stage : 1;
       for (int it = blockIdx.x; it < a.n_items; it += gridDim.x) {
         const int nb = it / n_tiles, tile = it - nb * n_tiles;
         const int tw = tile % a.nW, th = (tile / a.nW) % a.nH, ti = tile / (a.nW * a.nH);
@@ -124,6 +144,24 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
             const int wc = strided ? w0 + (tb == 0 ? -1 : 0) : w0 - 1 + tb;
             const int c_base = strided ? (tb == 1 ? 0 : a.C) : 0;
             int c_off = 0;
+            if constexpr (RW) {
+              // a stage holds the boxes of `tps` consecutive taps: it is opened by its first
+              // tap and advanced after its last
+              const int in_stage = tap % tps;
+              const uint32_t fb = bar_full + 8u * s;
+              if (in_stage == 0) {
+                if (issued >= n_stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
+                ++issued;
+                mbar_expect_tx(fb, stage_bytes);
+              }
+              uint32_t sa = ring + (uint32_t)s * stage_bytes + (uint32_t)(in_stage * kblocks) * a_bytes;
+              for (int kb = 0; kb < kblocks; ++kb, c_off += cb, sa += a_bytes) {
+                if (!strided) tma_load_4d(sa, &mapX, fb, c_off, wc, hc, i0);
+                else tma_load_5d(sa, &mapX, fb, c_base + c_off, wc, prow, hc, i0);
+              }
+              if (in_stage == tps - 1 && ++s == n_stages) { s = 0; ph ^= 1u; }
+              continue;
+            }
             for (int kb = 0; kb < kblocks; ++kb, c_off += cb) {
               if (issued >= n_stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
               ++issued;
@@ -148,7 +186,10 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
     const int ksteps = a.cB / 32;
     int s = 0; uint32_t ph = 0;
     int li = 0;
-    for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
+    bool w_ok = true;
+    if constexpr (RW) w_ok = __all_sync(0xffffffffu, mbar_wait(bar_w, 0u, abort_p));
+    if (!w_ok) *abort_p = 1u;
+    for (int it = blockIdx.x; it < a.n_items && w_ok; it += gridDim.x, ++li) {
       const int buf = li & 1;
       const uint32_t aph = (uint32_t)(li >> 1) & 1u;
       bool ok = __all_sync(0xffffffffu, mbar_wait(bar_acc_empty + 8u * buf, aph ^ 1u, abort_p));
@@ -157,6 +198,23 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
       for (int st = 0; st < steps && ok; ++st) {
         if (!__all_sync(0xffffffffu, mbar_wait(bar_full + 8u * s, ph, abort_p))) { ok = false; break; }
         tc_fence_after();
+        if constexpr (RW) {
+          // the stage's boxes in tap order against the resident slices of the same taps
+          const int per_stage = a.taps_per_stage * a.KB;
+          uint32_t sa = ring + (uint32_t)s * stage_bytes;
+          uint32_t sb = base + (uint32_t)(st * per_stage) * b_bytes;
+          for (int j = 0; j < per_stage; ++j, sa += a_bytes, sb += b_bytes) {
+            const uint64_t da = a.cB == 128 ? make_desc_sw128(sa) : desc_sw64(sa);
+            const uint64_t db = a.cB == 128 ? make_desc_sw128(sb) : desc_sw64(sb);
+            if (leader)
+              for (int k = 0; k < ksteps; ++k)
+                mma_i8(tacc, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (st | j | k) != 0 ? 1u : 0u);
+          }
+          if (leader) mma_commit(bar_empty + 8u * s);
+          __syncwarp();
+          if (++s == a.stages) { s = 0; ph ^= 1u; }
+          continue;
+        }
         const uint32_t sa = base + (uint32_t)s * stage_bytes;
         const uint64_t da = a.cB == 128 ? make_desc_sw128(sa) : desc_sw64(sa);
         const uint64_t db = a.cB == 128 ? make_desc_sw128(sa + a_bytes) : desc_sw64(sa + a_bytes);
@@ -250,14 +308,27 @@ __global__ void __launch_bounds__(kDtThreads, 1)
 k_direct_conv_tc(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
                  const DirectTcArgs a, const float* __restrict__ bias, void* __restrict__ y,
                  int* __restrict__ status) {
-  direct_conv_tc_body<false>(mapX, mapW, a, bias, y, status);
+  direct_conv_tc_body<false, false>(mapX, mapW, a, bias, y, status);
+}
+__global__ void __launch_bounds__(kDtThreads, 1)
+k_direct_conv_tc_resident(const __grid_constant__ CUtensorMap mapX, const __grid_constant__ CUtensorMap mapW,
+                          const DirectTcArgs a, const float* __restrict__ bias, void* __restrict__ y,
+                          int* __restrict__ status) {
+  direct_conv_tc_body<false, true>(mapX, mapW, a, bias, y, status);
+}
+__global__ void __launch_bounds__(kDtThreads, 1)
+k_direct_conv_tc_resident_per_channel(const __grid_constant__ CUtensorMap mapX,
+                                      const __grid_constant__ CUtensorMap mapW, const DirectTcArgs a,
+                                      const float* __restrict__ bias, void* __restrict__ y,
+                                      int* __restrict__ status) {
+  direct_conv_tc_body<true, true>(mapX, mapW, a, bias, y, status);
 }
 __global__ void __launch_bounds__(kDtThreads, 1)
 k_direct_conv_tc_per_channel(const __grid_constant__ CUtensorMap mapX,
                              const __grid_constant__ CUtensorMap mapW, const DirectTcArgs a,
                              const float* __restrict__ bias, void* __restrict__ y,
                              int* __restrict__ status) {
-  direct_conv_tc_body<true>(mapX, mapW, a, bias, y, status);
+  direct_conv_tc_body<true, false>(mapX, mapW, a, bias, y, status);
 }
 
 // One status word per device for the plan-less direct convolution.
@@ -287,9 +358,25 @@ DirectTcArgs direct_tc_geometry(int N, int C, int H_in, int W_in, int K, int str
   while (a.BN > 64 && tiles * (K / a.BN) < (num_sms * 4) / 5) a.BN /= 2;
   a.n_nblk = K / a.BN;
   a.n_items = tiles * a.n_nblk;
-  const size_t stage = (size_t)128 * a.cB + (size_t)a.BN * a.cB;
+  const size_t a_bytes = (size_t)128 * a.cB, b_bytes = (size_t)a.BN * a.cB;
+  const size_t stage = a_bytes + b_bytes;
   a.stages = (int)((192 * 1024) / stage);
   if (a.stages > 8) a.stages = 8;
+  // resident weights: one block of output channels, and room for at least three stages of
+  // three taps each beside them (with less room the shallower ring costs more than the saved
+  // copies gain: 19.1 against 17.8 us on the 128-channel 16x16 layer at batch 256)
+  const size_t budget = 200 * 1024, res = 9 * (size_t)a.KB * b_bytes;
+  const size_t st3 = 3 * (size_t)a.KB * a_bytes;
+  a.w_resident = 0;
+  a.taps_per_stage = 1;
+  // (a whole item, nine taps, per stage leaves two stages: 46 us on the 64-channel 32x32
+  // layer against 35 with three taps per stage and six stages)
+  if (a.n_nblk == 1 && res + 3 * st3 <= budget) {
+    a.w_resident = 1;
+    a.taps_per_stage = 3;
+    a.stages = (int)((budget - res) / st3);
+    if (a.stages > 8) a.stages = 8;
+  }
   int acc_stride = 32;
   while (acc_stride < a.BN) acc_stride *= 2;
   a.acc_stride = acc_stride;
@@ -317,20 +404,22 @@ int launch_direct_conv_tc(const DirectTcArgs& a, int device, int num_sms, const 
                           const CUtensorMap& mapW, const float* bias, void* y, cudaStream_t st) {
   int* status = direct_tc_status_word(device);
   if (status == nullptr) return -5;
-  const size_t stage = (size_t)128 * a.cB + (size_t)a.BN * a.cB;
+  const size_t a_bytes = (size_t)128 * a.cB, b_bytes = (size_t)a.BN * a.cB;
+  const size_t ring = a.w_resident
+                          ? 9 * (size_t)a.KB * b_bytes + (size_t)a.stages * a.taps_per_stage * a.KB * a_bytes
+                          : (size_t)a.stages * (a_bytes + b_bytes);
   const bool pk = a.s_w_K != nullptr || a.s_Y_K != nullptr;
-  const size_t smem = 1024 + (size_t)a.stages * stage + (size_t)a.K * (pk ? 8 : 4) + 16 * (size_t)a.stages + 64;
+  const size_t smem = 1024 + ring + (size_t)a.K * (pk ? 8 : 4) + 16 * (size_t)a.stages + 64;
   const int grid = a.n_items < num_sms ? a.n_items : num_sms;
-  if (pk) {
-    static DeviceOnce once_pk;
-    if (int rc = set_max_smem(once_pk, device, k_direct_conv_tc_per_channel, 227 * 1024)) return rc;
-    return launch_kernel(k_direct_conv_tc_per_channel, dim3((unsigned)grid), dim3(kDtThreads), smem, st,
-                         true, mapX, mapW, a, bias, y, status);
-  }
-  static DeviceOnce once;
-  if (int rc = set_max_smem(once, device, k_direct_conv_tc, 227 * 1024)) return rc;
-  return launch_kernel(k_direct_conv_tc, dim3((unsigned)grid), dim3(kDtThreads), smem, st, true, mapX, mapW,
-                       a, bias, y, status);
+  auto go = [&](auto kernel, DeviceOnce& once) -> int {
+    if (int rc = set_max_smem(once, device, kernel, 227 * 1024)) return rc;
+    return launch_kernel(kernel, dim3((unsigned)grid), dim3(kDtThreads), smem, st, true, mapX, mapW, a,
+                         bias, y, status);
+  };
+  static DeviceOnce once, once_pk, once_rw, once_rw_pk;
+  if (a.w_resident) return pk ? go(k_direct_conv_tc_resident_per_channel, once_rw_pk)
+                              : go(k_direct_conv_tc_resident, once_rw);
+  return pk ? go(k_direct_conv_tc_per_channel, once_pk) : go(k_direct_conv_tc, once);
 }
 
 }  // namespace wino

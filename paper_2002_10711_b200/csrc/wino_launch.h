@@ -146,6 +146,10 @@ struct DirectTcArgs {
   int cB, KB;              // channel bytes per stage (64 or 128) and stages per tap
   int stages, tmem_cols, acc_stride;
   int n_items;
+  // Narrow layers whose whole weight tensor fits beside the input ring: the weights are
+  // fetched once per block and stay in shared memory (w_resident), and a stage then holds the
+  // input boxes of `taps_per_stage` = 3 taps, one row of the filter (1 otherwise).
+  int w_resident, taps_per_stage;
   float mult, s_in, s_Y, lo_Y, hi_Y;
   int z_Y, out_dtype;
   // per-output-channel scales (device arrays of K floats, nullable) and the per-layer scales

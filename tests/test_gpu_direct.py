@@ -29,6 +29,7 @@ def _run(N, C, H, W, K, stride, q_x, q_w, q_Y, x_q, w_q, bias, out_dtype=0):
                                    (1, 20, 6, 11, 12),
                                    (3, 128, 8, 8, 64), (5, 64, 4, 4, 96), (1, 256, 5, 19, 32), (2, 192, 1, 1, 64),
                                    (1, 512, 4, 4, 512), (2, 64, 9, 7, 32),
+                                   (2, 128, 7, 9, 32), (20, 64, 16, 16, 64),   # weights resident in shared memory, several items per block
                                    (2, 3, 32, 32, 64), (2, 5, 7, 9, 6)])   # any channel count: byte-wise kernel
 @pytest.mark.parametrize("stride", [1, 2])
 @pytest.mark.parametrize("variant", ["plain", "relu_bias", "zero_points"])
@@ -142,6 +143,7 @@ def test_direct_conv_argument_checks():
 # per-output-channel scales (Section 7) on every direct-convolution kernel: tensor cores
 # (stride 1 and 2), integer dot products, byte-wise
 @pytest.mark.parametrize("shape,stride", [((2, 64, 9, 7, 32), 1), ((3, 128, 8, 8, 64), 2), ((1, 256, 5, 19, 288), 1),
+                                          ((20, 64, 16, 16, 64), 2), ((2, 128, 7, 9, 32), 1),
                                           ((2, 16, 9, 7, 8), 1), ((1, 20, 6, 11, 12), 2), ((2, 3, 16, 16, 6), 1)])
 @pytest.mark.parametrize("which", ["both", "weights_only", "output_only"])
 @pytest.mark.parametrize("out_dtype", [0, 1])
