@@ -129,10 +129,24 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
             tma_load_3d(dst, &mapW, bar_w, kb * cb, tap, 0);
       }
       const int tps = RW ? a.taps_per_stage : 1;
+      // item -> (channel block, tile column, tile row, image group): divided out once, then
+      // advanced by the grid's stride with carries (an integer division costs this thread some
+      // forty instructions, and narrow layers have a dozen items per block)
+      const int nW = a.nW, nH = a.nH, nI = a.nI;
+      int nb = (int)blockIdx.x / n_tiles;
+      int tw, th, ti;
+      {
+        const int tile = (int)blockIdx.x - nb * n_tiles;
+        tw = tile % nW; th = (tile / nW) % nH; ti = tile / (nW * nH);
+      }
+      const int step_nb = (int)gridDim.x / n_tiles, step_r = (int)gridDim.x - step_nb * n_tiles;
+      const int d_w = step_r % nW, d_h = (step_r / nW) % nH, d_i = step_r / (nW * nH);
+      int in_stage = 0;
       for (int it = blockIdx.x; it < a.n_items; it += gridDim.x) {
-        const int nb = it / n_tiles, tile = it - nb * n_tiles;
-        const int tw = tile % a.nW, th = (tile / a.nW) % a.nH, ti = tile / (a.nW * a.nH);
         const int w0 = tw * a.BW, h0 = th * a.BH, i0 = ti * a.BI, k_row = nb * a.BN;
+        tw += d_w; if (tw >= nW) { tw -= nW; ++th; }
+        th += d_h; if (th >= nH) { th -= nH; ++ti; }
+        ti += d_i; nb += step_nb; if (ti >= nI) { ti -= nI; ++nb; }
         bool ok = true;
         int tap = 0;
         for (int ta = 0; ta < 3 && ok; ++ta) {
@@ -147,7 +161,6 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
             if constexpr (RW) {
               // a stage holds the boxes of `tps` consecutive taps: it is opened by its first
               // tap and advanced after its last
-              const int in_stage = tap % tps;
               const uint32_t fb = bar_full + 8u * s;
               if (in_stage == 0) {
                 if (issued >= n_stages && !mbar_wait(bar_empty + 8u * s, ph ^ 1u, abort_p)) { ok = false; break; }
@@ -159,7 +172,10 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
                 if (!strided) tma_load_4d(sa, &mapX, fb, c_off, wc, hc, i0);
                 else tma_load_5d(sa, &mapX, fb, c_base + c_off, wc, prow, hc, i0);
               }
-              if (in_stage == tps - 1 && ++s == n_stages) { s = 0; ph ^= 1u; }
+              if (++in_stage == tps) {
+                in_stage = 0;
+                if (++s == n_stages) { s = 0; ph ^= 1u; }
+              }
               continue;
             }
             for (int kb = 0; kb < kblocks; ++kb, c_off += cb) {
@@ -369,8 +385,10 @@ DirectTcArgs direct_tc_geometry(int N, int C, int H_in, int W_in, int K, int str
   const size_t st3 = 3 * (size_t)a.KB * a_bytes;
   a.w_resident = 0;
   a.taps_per_stage = 1;
-  // (a whole item, nine taps, per stage leaves two stages: 46 us on the 64-channel 32x32
-  // layer against 35 with three taps per stage and six stages)
+  // (a whole item, nine taps, per stage measured the same as three: 36.2 against 36.6 us on
+  // the 64-channel 32x32 layer.  What then bounds these layers is the rate at which the copy
+  // engine delivers box rows, about one per two cycles per SM whatever their width, and
+  // 64-channel rows are 64 bytes)
   if (a.n_nblk == 1 && res + 3 * st3 <= budget) {
     a.w_resident = 1;
     a.taps_per_stage = 3;
