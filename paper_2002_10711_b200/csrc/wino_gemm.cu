@@ -110,10 +110,26 @@ __device__ __forceinline__ float acc_to_float(uint32_t v) {
 // Epilogue of one 32-column chunk of one accumulator row.  FULL: all 32 columns
 // are inside K (no per-element guards).  STATS: track max |M| for calibration.  PK: the
 // multiplier of Q_M varies per output channel (column).
-template <bool SMALL, bool FULL, bool STATS, bool PK>
+template <bool SMALL, bool FULL, bool STATS, bool PK, bool LEAN = false>
 __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (&r)[32], int k0,
                                                long o, int out_mode, void* out, float& vmax,
                                                bool wide_store, const float* mult_k) {
+  if constexpr (LEAN) {
+    // the one configuration the lean kernel is launched for: int8 codes, upper bound 127
+    // (saturating pack), 32-byte aligned rows
+    const float lo_m = __fadd_rn(p.lo_M, kMagic), hi_m = __fadd_rn(p.hi_M, kMagic);
+    uint32_t w[8];
+#pragma unroll
+    for (int q = 0; q < 8; ++q)
+      w[q] = quant_pack4<true>(acc_to_float<SMALL>(r[4 * q + 0]), acc_to_float<SMALL>(r[4 * q + 1]),
+                               acc_to_float<SMALL>(r[4 * q + 2]), acc_to_float<SMALL>(r[4 * q + 3]),
+                               p.mult_M, lo_m, hi_m);
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(
+                     reinterpret_cast<int8_t*>(out) + o),
+                 "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7])
+                 : "memory");
+    return;
+  }
   if constexpr (STATS) {
 #pragma unroll
     for (int j = 0; j < 32; ++j)
@@ -176,7 +192,7 @@ __device__ __forceinline__ void epilogue_chunk(const Params& p, const uint32_t (
 }
 
 // The epilogue warps' loop over their work items.
-template <bool SMALL, bool FULL, bool STATS, bool PK = false>
+template <bool SMALL, bool FULL, bool STATS, bool PK = false, bool LEAN = false>
 __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs& a, void* out,
                                               unsigned* absmaxM, uint32_t tmem_base,
                                               uint32_t bar_acc_full, uint32_t bar_acc_empty,
@@ -203,17 +219,20 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
     // the accumulator holds MB blocks of BN columns side by side; one chunk at a
     // time per warp, the four warps of a scheduler hide each other's
     // tensor-memory load latency
+    auto chunk = [&](const uint32_t (&r)[32], int col) {
+      const int j = a.MB > 1 ? col / a.BN : 0;
+      const int kcol = col - j * a.BN;
+      const int tau = (mb * a.MB + j) * kBM + quad * 32 + lane;
+      if (tau >= p.T) return;
+      const int k0 = nb * a.BN + kcol;
+      const long o = ((long)xi * p.T + tau) * p.K + k0;
+      epilogue_chunk<SMALL, FULL, STATS, PK, LEAN>(p, r, k0, o, a.out_mode, out, vmax, a.wide_store != 0, mult_k);
+    };
     for (int col = sub * 32; col < a.MB * a.BN; col += 128) {
       uint32_t r0[32];
       tmem_ld32(tacc + (uint32_t)col, r0);
       tmem_ld_wait();
-      const int j = a.MB > 1 ? col / a.BN : 0;
-      const int kcol = col - j * a.BN;
-      const int tau = (mb * a.MB + j) * kBM + quad * 32 + lane;
-      if (tau >= p.T) continue;
-      const int k0 = nb * a.BN + kcol;
-      const long o = ((long)xi * p.T + tau) * p.K + k0;
-      epilogue_chunk<SMALL, FULL, STATS, PK>(p, r0, k0, o, a.out_mode, out, vmax, a.wide_store != 0, mult_k);
+      chunk(r0, col);
     }
     tc_fence_before();
     __syncwarp();
@@ -225,7 +244,10 @@ __device__ __forceinline__ void epilogue_loop(const Params& p, const GemmTcArgs&
 
 // PK: Q_M takes one multiplier per output channel (a build of its own, so that the
 // per-layer kernel carries none of that code).
-template <bool PK>
+// LEAN: only the epilogue of the common case is compiled in (Q_M to int8 codes with upper
+// bound 127, C <= 260, whole 32-column chunks, 32-byte aligned rows); the kernel's code is a
+// third of the general one's, which shows at every launch.
+template <bool PK, bool LEAN = false>
 __device__ __forceinline__ void gemm_tc_body(const Params& p, const CUtensorMap* mapV,
                                              const CUtensorMap* mapU, const GemmTcArgs& a,
                                              void* __restrict__ out, unsigned* __restrict__ absmaxM,
@@ -415,7 +437,11 @@ __device__ __forceinline__ void gemm_tc_body(const Params& p, const CUtensorMap*
       mult_k = tab;
     }
     griddep_wait();
-    if constexpr (PK) {
+    if constexpr (LEAN) {
+      (void)per_channel; (void)small; (void)full;
+      epilogue_loop<true, true, false, false, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
+                                                    bar_acc_empty, abort_p, warp, lane, trace_step);
+    } else if constexpr (PK) {
       (void)per_channel;
       if (absmaxM != nullptr)
         epilogue_loop<false, false, true, true>(p, a, out, absmaxM, tmem_base, bar_acc_full,
@@ -455,6 +481,12 @@ k_gemm_tc(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap 
           const __grid_constant__ CUtensorMap mapU, const GemmTcArgs a, void* __restrict__ out,
           unsigned* __restrict__ absmaxM, int* __restrict__ status) {
   gemm_tc_body<false>(p, &mapV, &mapU, a, out, absmaxM, status);
+}
+__global__ void __launch_bounds__(kGemmThreads, 1)
+k_gemm_tc_lean(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV,
+               const __grid_constant__ CUtensorMap mapU, const GemmTcArgs a, void* __restrict__ out,
+               unsigned* __restrict__ absmaxM, int* __restrict__ status) {
+  gemm_tc_body<false, true>(p, &mapV, &mapU, a, out, absmaxM, status);
 }
 __global__ void __launch_bounds__(kGemmThreads, 1)
 k_gemm_tc_per_channel(const __grid_constant__ Params p, const __grid_constant__ CUtensorMap mapV,
@@ -511,6 +543,14 @@ int launch_gemm_tc(const Params& p, const LaunchOpt& o, const TcGeom& g, const C
     const size_t smem = g.smem + (a.chan_smem ? (size_t)p.K * 4 : 0);
     return launch_kernel(k_gemm_tc_per_channel, dim3((unsigned)g.grid), dim3(kGemmThreads), smem, st,
                          o.pdl, p, mapV, mapU, a, out, absmaxM, status);
+  }
+  const bool lean = absmaxM == nullptr && out_mode == kOutMq && p.hi_M == 127.0f && a.wide_store &&
+                    p.C <= 260 && p.K % a.BN == 0 && a.BN % 32 == 0;
+  if (lean) {
+    static DeviceOnce once_lean;
+    if (int rc = set_max_smem(once_lean, o.device, k_gemm_tc_lean, 227 * 1024)) return rc;
+    return launch_kernel(k_gemm_tc_lean, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl,
+                         p, mapV, mapU, a, out, absmaxM, status);
   }
   return launch_kernel(k_gemm_tc, dim3((unsigned)g.grid), dim3(kGemmThreads), g.smem, st, o.pdl, p,
                        mapV, mapU, a, out, absmaxM, status);
