@@ -377,6 +377,15 @@ __device__ __forceinline__ void gemm_tc_body(const Params& p, const CUtensorMap*
     // values; one elected lane issues the MMAs and the commits.
     const bool leader = elect_one();
     const uint32_t idesc = make_idesc_i8(kBM, a.BN);
+    // What does not change from stage to stage is computed once: this warp's every
+    // instruction costs ten to twenty cycles and a stage's MMAs take five hundred.  Descriptors
+    // are linear in the tile address (units of 16 bytes), so a stage's are the first stage's
+    // plus a multiple of the stage size.
+    const uint64_t da_first = make_desc_sw128(base);
+    const uint32_t stage_units = stage_bytes >> 4, a_units = a_bytes >> 4;
+    const uint32_t b_units = (uint32_t)a.MB * a_units;
+    const int last_ksteps = (p.C - (KB - 1) * kStageK + 31) / 32;   // 1..4
+    uint32_t s_units = 0;   // s * stage_units
     int s = 0; uint32_t ph = 0;
     int li = 0;
     for (int it = blockIdx.x; it < a.n_items; it += gridDim.x, ++li) {
@@ -392,12 +401,11 @@ __device__ __forceinline__ void gemm_tc_body(const Params& p, const CUtensorMap*
         if (leader && li == 1 && kb == 0) WINO_ST(g_gemm_trace, trace_step, 10);
         if (leader && li == 1 && kb == KB - 1) WINO_ST(g_gemm_trace, trace_step, 11);
         tc_fence_after();
-        const uint32_t sa = base + (uint32_t)s * stage_bytes;
-        const uint64_t db = make_desc_sw128(sa + (uint32_t)a.MB * a_bytes);
-        const int remc = p.C - kb * kStageK;
-        const int ksteps = remc >= kStageK ? 4 : (remc + 31) / 32;
+        const uint64_t da0 = da_first + s_units;
+        const uint64_t db = da0 + b_units;
+        const int ksteps = kb == KB - 1 ? last_ksteps : 4;
         for (int j = 0; j < a.MB; ++j) {
-          const uint64_t da = make_desc_sw128(sa + (uint32_t)j * a_bytes);
+          const uint64_t da = da0 + (uint64_t)(j * (int)a_units);
           const uint32_t td = tacc + (uint32_t)(j * a.BN);
           if (leader) {
             if (ksteps == 4) {
@@ -413,7 +421,8 @@ __device__ __forceinline__ void gemm_tc_body(const Params& p, const CUtensorMap*
         }
         if (leader) mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
         __syncwarp();
-        if (++s == a.stages) { s = 0; ph ^= 1u; }
+        s_units += stage_units;
+        if (++s == a.stages) { s = 0; s_units = 0; ph ^= 1u; }
       }
       if (!ok) { *abort_p = 1u; break; }
       if (leader) mma_commit(bar_acc_full + 8u * buf);  // accumulator complete
