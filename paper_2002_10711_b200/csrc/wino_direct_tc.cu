@@ -200,6 +200,12 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
     const bool leader = elect_one();
     const uint32_t idesc = make_idesc_i8(128, a.BN);
     const int ksteps = a.cB / 32;
+    // descriptors are linear in the tile address (units of 16 bytes): the first tile's, once,
+    // plus running offsets, instead of rebuilding them in every stage
+    const uint64_t d_first = a.cB == 128 ? make_desc_sw128(base) : desc_sw64(base);
+    const uint32_t a_units = a_bytes >> 4, b_units = b_bytes >> 4, stage_units = stage_bytes >> 4;
+    const uint32_t ring_units = (ring - base) >> 4;
+    uint32_t s_units = 0;   // s * stage_units
     int s = 0; uint32_t ph = 0;
     int li = 0;
     bool w_ok = true;
@@ -217,30 +223,29 @@ __device__ __forceinline__ void direct_conv_tc_body(const CUtensorMap& mapX, con
         if constexpr (RW) {
           // the stage's boxes in tap order against the resident slices of the same taps
           const int per_stage = a.taps_per_stage * a.KB;
-          uint32_t sa = ring + (uint32_t)s * stage_bytes;
-          uint32_t sb = base + (uint32_t)(st * per_stage) * b_bytes;
-          for (int j = 0; j < per_stage; ++j, sa += a_bytes, sb += b_bytes) {
-            const uint64_t da = a.cB == 128 ? make_desc_sw128(sa) : desc_sw64(sa);
-            const uint64_t db = a.cB == 128 ? make_desc_sw128(sb) : desc_sw64(sb);
+          uint64_t da = d_first + (ring_units + s_units);
+          uint64_t db = d_first + (uint32_t)(st * per_stage) * b_units;
+          for (int j = 0; j < per_stage; ++j, da += a_units, db += b_units) {
             if (leader)
               for (int k = 0; k < ksteps; ++k)
                 mma_i8(tacc, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (st | j | k) != 0 ? 1u : 0u);
           }
           if (leader) mma_commit(bar_empty + 8u * s);
           __syncwarp();
-          if (++s == a.stages) { s = 0; ph ^= 1u; }
+          s_units += stage_units;
+          if (++s == a.stages) { s = 0; s_units = 0; ph ^= 1u; }
           continue;
         }
-        const uint32_t sa = base + (uint32_t)s * stage_bytes;
-        const uint64_t da = a.cB == 128 ? make_desc_sw128(sa) : desc_sw64(sa);
-        const uint64_t db = a.cB == 128 ? make_desc_sw128(sa + a_bytes) : desc_sw64(sa + a_bytes);
+        const uint64_t da = d_first + s_units;
+        const uint64_t db = da + a_units;
         if (leader) {
           for (int k = 0; k < ksteps; ++k)
             mma_i8(tacc, da + (uint64_t)(k * 2), db + (uint64_t)(k * 2), idesc, (st | k) != 0 ? 1u : 0u);
           mma_commit(bar_empty + 8u * s);   // frees the stage when these MMAs retire
         }
         __syncwarp();
-        if (++s == a.stages) { s = 0; ph ^= 1u; }
+        s_units += stage_units;
+        if (++s == a.stages) { s = 0; s_units = 0; ph ^= 1u; }
       }
       if (!ok) { *abort_p = 1u; break; }
       if (leader) mma_commit(bar_acc_full + 8u * buf);  // accumulator complete
