@@ -173,8 +173,9 @@ __device__ __forceinline__ void bulk_prefetch_l2(const void* gptr, uint32_t byte
 // This block's share of a buffer that the whole grid is asked to bring into L2.
 __device__ __forceinline__ void l2_hint_slice(const uint8_t* base, uint32_t total_bytes) {
   if (base == nullptr) return;
-  const uint32_t per = ((total_bytes + gridDim.x - 1) / gridDim.x + 15u) & ~15u;
-  const uint32_t off = blockIdx.x * per;
+  const uint32_t blocks = gridDim.x * gridDim.y, block = blockIdx.y * gridDim.x + blockIdx.x;
+  const uint32_t per = ((total_bytes + blocks - 1) / blocks + 15u) & ~15u;
+  const uint32_t off = block * per;
   if (off < total_bytes) bulk_prefetch_l2(base + off, min(per, total_bytes - off));
 }
 __device__ __forceinline__ void tma_prefetch_l2_3d(const CUtensorMap* map, int c0, int c1, int c2) {
