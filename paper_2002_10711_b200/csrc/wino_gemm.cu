@@ -517,7 +517,10 @@ TcGeom tc_geometry(const Params& p, int num_sms) {
   const size_t per_stage = (size_t)g.MB * kBM * kStageK + (size_t)g.BN * kStageK;
   g.stages = (int)((196 * 1024) / per_stage);
   const int KB = (p.C + kStageK - 1) / kStageK;
-  if (g.stages > 2 * KB) g.stages = 2 * KB;   // two items' worth is all the ring can use
+  // one and a half items' worth: with two whole items in the ring the second item's operands
+  // compete with the first item's for the path from L2 and delay its accumulator (cfg3: 5.87 us
+  // with four stages, 5.74 with three, 6.12 with two)
+  if (g.stages > (3 * KB + 1) / 2) g.stages = (3 * KB + 1) / 2;
   if (g.stages > 8) g.stages = 8;
   if (g.stages < 1) g.stages = 1;
   int acc_stride = 32;
